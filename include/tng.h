@@ -1,0 +1,182 @@
+/*
+ * tng.h -- C ABI of libtng: the data-parallel hot path of Trajectory Normalized
+ * Gradients (TNG, arXiv 1901.08227) on one NVIDIA B200 (sm_100a).
+ *
+ * One round (Algorithm 1 of the paper, with Eq. 2 / Eq. 3 of Section 3):
+ *   fuse the ring of past aggregated vectors into a shared reference r
+ *   -> normalise every worker's gradient against r (g - r, or g ./ r)
+ *   -> compress it (stochastic sign / ternary / s-level quantiser, per-block scale)
+ *   -> [the packed codes + scales are the "wire"]
+ *   -> decode all M workers, average, add (or multiply) the reference back
+ *   -> push the result into the ring.
+ * M workers are simulated as a batch: worker m's gradient is row m of `grads`.
+ *
+ * Conventions
+ *   - `*_dev` pointers are CUDA device pointers, `*_host` pointers host memory.
+ *     Device vectors must be 16-byte aligned; a row stride `ld` (in floats) must
+ *     be a multiple of 4 and >= d.  Violations return TNG_ERR_INVALID_ARG.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls
+ *     only enqueue work unless stated otherwise.
+ *   - The caller owns every buffer it passes.  The library owns the tng_ctx and,
+ *     unless a workspace is bound, one device allocation it frees in tng_destroy.
+ *   - No call aborts or throws; every failure is a tng_status.  There is no CPU
+ *     fallback: without a CUDA device the calls that touch the GPU return TNG_ERR_CUDA.
+ *   - A context is not thread-safe; use it from one host thread at a time and with one
+ *     stream at a time.
+ */
+#ifndef TNG_H
+#define TNG_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tng_ctx tng_ctx;
+
+typedef enum {
+    TNG_OK = 0,
+    TNG_ERR_INVALID_ARG = 1, /* bad size, enum, alignment, NULL pointer */
+    TNG_ERR_STATE = 2,       /* call not allowed now (options after the first round, ...) */
+    TNG_ERR_ALLOC = 3,       /* device or host allocation failed / workspace too small */
+    TNG_ERR_CUDA = 4,        /* a CUDA call or launch failed; tng_last_cuda_error() has the code */
+    TNG_ERR_NONFINITE = 5,   /* a NaN/Inf block scale was produced in an earlier round */
+    TNG_ERR_UNSUPPORTED = 6
+} tng_status;
+
+/* value = bits per coordinate symbol */
+typedef enum { TNG_CODEC_SIGN1 = 1, TNG_CODEC_TERN2 = 2, TNG_CODEC_QSGD4 = 4 } tng_codec;
+typedef enum { TNG_NORM_NONE = 0, TNG_NORM_DIFF = 1, TNG_NORM_QUOT = 2 } tng_norm_mode;
+typedef enum {
+    TNG_FUSE_AUTO = 0,     /* K == 1 -> LAST, else LSQ */
+    TNG_FUSE_LAST = 1,     /* r = newest aggregate (delayed gradient, Sec. 3.1 / Sec. 4.2 protocol) */
+    TNG_FUSE_MEAN = 2,     /* r = window average of the k stored aggregates (Sec. 3.1) */
+    TNG_FUSE_LSQ = 3,      /* r = sum_j alpha_j h_j minimising sum_m ||g^m - r||^2 (C_nz of Prop. 2) */
+    TNG_FUSE_HINDSIGHT = 4 /* alpha from the history alone: regress h_1 on h_2..h_k, shift by one */
+} tng_fuse_mode;
+
+typedef enum {
+    TNG_OPT_BLOCK = 0,       /* coordinates per scale; 0 = one scale per vector (the paper's R);
+                                otherwise a multiple of 128.  Default 128. */
+    TNG_OPT_QSGD_LEVELS = 1, /* s in 1..7 (TNG_CODEC_QSGD4 only).  Default 7. */
+    TNG_OPT_SCALE_KIND = 2,  /* 0 = max|v| (Sec. 3.2), 1 = L2 norm of the block.  Default 0. */
+    TNG_OPT_SEED_LO = 3,     /* low / high 32 bits of the Philox key.  Default 0. */
+    TNG_OPT_SEED_HI = 4,
+    TNG_OPT_FUSE_MODE = 5,   /* a tng_fuse_mode.  Default TNG_FUSE_AUTO. */
+    TNG_OPT_RIDGE = 6,       /* relative ridge of the K x K solve.  Default 1e-6. */
+    TNG_OPT_QUOT_EPS = 7,    /* floor of |r| relative to its tile maximum, quotient form.  Default 2^-4. */
+    TNG_OPT_TIMING = 8,      /* 1 = record CUDA events around every stage of tng_step.  Default 0. */
+    TNG_OPT_HOST_STAGING = 9 /* 1 = reserve device staging so tng_step_host can be used.  Default 0. */
+} tng_option;
+
+#define TNG_MAX_WORKERS 64
+#define TNG_MAX_HISTORY 16
+#define TNG_TILE 128 /* coordinates per wire tile */
+
+/* Plain-old-data snapshot filled by tng_stats. */
+typedef struct {
+    uint64_t d;
+    uint32_t M, K;
+    uint32_t k;              /* history vectors currently stored */
+    uint32_t fuse_mode;      /* effective mode (never AUTO) */
+    uint64_t rounds;         /* completed rounds (the Philox step counter) */
+    double bits_per_coord;   /* b + 32/B + 64 K/d */
+    double alpha[TNG_MAX_HISTORY];                     /* coefficients of the last fusion */
+    double gram[TNG_MAX_HISTORY * TNG_MAX_HISTORY];    /* k x k, row-major (LSQ / HINDSIGHT) */
+    double rhs[TNG_MAX_HISTORY];                       /* <h_i, mean gradient> */
+    double grad_sq;          /* (1/M) sum_m ||g^m||^2 of the last fusion */
+    double cnz;              /* estimate of C_nz = sum_m||g^m - r||^2 / sum_m||g^m||^2; NaN if unknown */
+    uint32_t solver_fallback;   /* 1 = last solve hit a bad pivot and used alpha = e_1 */
+    uint32_t reserved;
+    uint64_t nonfinite_scales;  /* block scales that were NaN/Inf since creation */
+    uint64_t kernel_launches;   /* kernels launched by this context since creation */
+    /* mean milliseconds per round of each stage over the rounds timed so far
+       (TNG_OPT_TIMING = 1), and how many rounds that is */
+    uint64_t timed_rounds;
+    double ms_dots, ms_solve, ms_combine, ms_encode, ms_decode;
+} tng_stats_t;
+
+/* ---- lifetime --------------------------------------------------------------- */
+/* d >= 1 coordinates, 1 <= M <= 64 workers, ring depth 1 <= K <= 16.  Host only. */
+tng_status tng_create(tng_ctx** out, uint64_t d, uint32_t M, uint32_t K, tng_codec codec,
+                      tng_norm_mode norm);
+/* Waits for the context's last stream, frees what the library allocated.  NULL is allowed. */
+void tng_destroy(tng_ctx* ctx);
+/* Options can change until the workspace is sized (tng_workspace_bytes, tng_bind_workspace
+ * or the first call that touches the device); later: TNG_ERR_STATE. */
+tng_status tng_set_option(tng_ctx* ctx, tng_option key, double value);
+/* Device bytes the context needs (ring K*d, reference, codes, scales, reduction scratch). */
+tng_status tng_workspace_bytes(tng_ctx* ctx, size_t* bytes);
+/* Use caller-owned device memory (256-byte aligned, >= tng_workspace_bytes) instead of an
+ * internal cudaMalloc.  Must come before the first device call.  Contents are cleared lazily
+ * on `stream` of the first device call. */
+tng_status tng_bind_workspace(tng_ctx* ctx, void* dev_ptr, size_t bytes);
+
+/* ---- the round ------------------------------------------------------------- */
+/* Seed the ring with a vector (Sec. 4.2: "initialise the reference with a full gradient"). */
+tng_status tng_push_reference(tng_ctx* ctx, const float* vec_dev, void* stream);
+/* One round on M gradient rows (row m at grads_dev + m*ld).  Writes the decoded aggregate
+ * v_t (d floats) to agg_out_dev if it is not NULL; the aggregate is always stored as the
+ * newest ring entry (tng_history(ctx, 0, ...)). */
+tng_status tng_step(tng_ctx* ctx, const float* grads_dev, uint64_t ld, float* agg_out_dev,
+                    void* stream);
+/* Same round for host buffers: copies the M rows to device staging, runs the round, copies the
+ * aggregate back, all on `stream`; returns after the stream has finished.  Needs
+ * TNG_OPT_HOST_STAGING = 1.  Pinned host memory makes the copies asynchronous and fast. */
+tng_status tng_step_host(tng_ctx* ctx, const float* grads_host, uint64_t ld, float* agg_out_host,
+                         void* stream);
+
+/* ---- stage-level entry points (the same kernels tng_step launches) ---------- */
+/* Fusion: Gram/rhs statistics, K x K solve, reference combine -> the context's reference. */
+tng_status tng_fuse(tng_ctx* ctx, const float* grads_dev, uint64_t ld, void* stream);
+/* Normalise + scale + quantise + pack against ref_dev (NULL = the context's reference).
+ * `step` is the Philox step counter to use (tng_step passes the round number). */
+tng_status tng_encode(tng_ctx* ctx, const float* grads_dev, uint64_t ld, const float* ref_dev,
+                      uint32_t step, void* stream);
+/* Unpack M code streams, dequantise, average, de-normalise against ref_dev (NULL = context's).
+ * Writes out_dev (d floats); does not touch the ring. */
+tng_status tng_decode_aggregate(tng_ctx* ctx, const float* ref_dev, float* out_dev, void* stream);
+
+/* ---- borrowed views (valid until the next call that changes them) ---------- */
+/* Wire: codes[m] at codes_dev + m*words_per_worker (uint32), scales[m] at scales_dev +
+ * m*scales_per_worker.  Tile T = coordinates [128T,128T+128) owns 4b words; word c*b+p, bit j,
+ * is bit p of the symbol of coordinate 128T + 4j + c. */
+tng_status tng_wire(tng_ctx* ctx, const uint32_t** codes_dev, size_t* words_per_worker,
+                    const float** scales_dev, size_t* scales_per_worker);
+tng_status tng_reference(tng_ctx* ctx, const float** ref_dev);
+/* h_{j+1}: j = 0 is the newest stored aggregate; j < k. */
+tng_status tng_history(tng_ctx* ctx, uint32_t j, const float** vec_dev);
+
+/* Synchronises the context's last stream and fills *out. */
+tng_status tng_stats(tng_ctx* ctx, tng_stats_t* out);
+const char* tng_status_string(tng_status s);
+/* cudaError_t value of the last failing CUDA call seen by this context (0 if none). */
+int tng_last_cuda_error(const tng_ctx* ctx);
+
+/* ---- gradient producers of the synthetic workloads (Section 4) -------------- */
+/* l2-regularised logistic regression, labels in {-1,+1}:
+ *   grad = -(1/n) sum_i b_i a_i sigma(-b_i a_i.w) + lambda2 w.
+ * X_dev: n x d row-major (d % 4 == 0 not required; rows are read with scalar tails),
+ * scratch_dev: at least tng_logistic_scratch_floats(n, d) floats. */
+size_t tng_logistic_scratch_floats(uint64_t n, uint64_t d);
+tng_status tng_logistic_grad(const float* X_dev, const float* b_dev, uint64_t n, uint64_t d,
+                             const float* w_dev, float lambda2, float* grad_dev, float* scratch_dev,
+                             void* stream);
+/* loss = (1/n) sum_i log(1+exp(-b_i a_i.w)) + (lambda2/2)||w||^2, written to *loss_dev (double). */
+tng_status tng_logistic_loss(const float* X_dev, const float* b_dev, uint64_t n, uint64_t d,
+                             const float* w_dev, float lambda2, double* loss_dev, float* scratch_dev,
+                             void* stream);
+/* Extended, uncoupled Rosenbrock f(x) = sum_i 100 (x_{2i+1} - x_{2i}^2)^2 + (1 - x_{2i})^2 (d even):
+ * grads[m][i] = df/dx_i + noise[m][i] (noise_dev may be NULL), rows of stride ld. */
+tng_status tng_rosenbrock_grad(const float* x_dev, uint64_t d, const float* noise_dev, uint32_t M,
+                               uint64_t ld, float* grads_dev, void* stream);
+tng_status tng_rosenbrock_value(const float* x_dev, uint64_t d, double* value_dev, void* stream);
+/* w <- w - eta * v (the outer update of Eq. 1). */
+tng_status tng_sgd_update(float* w_dev, const float* v_dev, uint64_t d, float eta, void* stream);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TNG_H */

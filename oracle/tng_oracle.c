@@ -306,15 +306,15 @@ static uint32_t quant_sign1(float v, float R, float u) {
     return (u * R < thr) ? 1u : 0u;
 }
 /* s-level stochastic uniform quantiser (QSGD, Alistarh et al. 2017):
- * a = (|v|/R) s, level floor(a) or floor(a)+1 with probability frac(a), capped
- * at s.  symbol bits 0..2 = level, bit 3 = negative. */
+ * a = (|v|/R) s, level floor(a) or floor(a)+1 with probability frac(a).  Both
+ * scale kinds give |v| <= R, so a <= s and the level never exceeds s.
+ * symbol bits 0..2 = level, bit 3 = negative. */
 static uint32_t quant_qsgd4(float v, float R, float u, int s) {
     float q = fabsf(v) / R;
     float a = q * (float)s;
     float l = floorf(a);
     float f = a - l;
     int L = (int)l + ((u < f) ? 1 : 0);
-    if (L > s) L = s;
     uint32_t neg = (L > 0 && v < 0.0f) ? 1u : 0u;
     return (uint32_t)L | (neg << 3);
 }

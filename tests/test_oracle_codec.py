@@ -225,6 +225,28 @@ def test_l2_scale_value_and_tree_shape():
     _, sc = oracle.encode(v[None], None, NORM_NONE, CODEC_QSGD4, B=128, scale_kind=SCALE_L2)
     assert sc[0, 0] == np.sqrt(np.float32(1.0 + 2.0 ** -23))
     assert np.float32(np.float32(np.float32(1 + e * e) + e * e) + e * e) == 1.0
+    # ... and pairs neighbours, not elements half a block apart: squares (1, 1, h, 2.25h), h = 2^-24,
+    # give (1+1) + (h+2.25h) = 2 + 2^-22, while (1+h) + (1+2.25h) = 1 + (1+2h) = 2
+    v = np.array([1.0, 1.0, e, 1.5 * e] + [0.0] * 124, dtype=np.float32)
+    _, sc = oracle.encode(v[None], None, NORM_NONE, CODEC_QSGD4, B=128, scale_kind=SCALE_L2)
+    assert sc[0, 0] == np.sqrt(np.float32(2.0 + 2.0 ** -22))
+    # two tiles in one block: the tree runs over the whole block
+    v2 = np.concatenate([v, v])
+    _, sc = oracle.encode(v2[None], None, NORM_NONE, CODEC_QSGD4, B=256, scale_kind=SCALE_L2)
+    assert sc[0, 0] == np.sqrt(np.float32(2 * np.float32(2.0 + 2.0 ** -22)))
+
+
+def test_zero_elements_never_fire_even_for_tiny_scales():
+    # P(z_d = 1) = |v_d| / R = 0 for v_d = 0, whatever u is: with the smallest
+    # subnormal as R, u * R rounds to zero for half of all u
+    tiny = np.float32(1.4e-45)
+    v = np.zeros(512, dtype=np.float32)
+    v[::128] = tiny
+    for codec in (CODEC_TERN2, CODEC_QSGD4):
+        for t in range(3):
+            codes, sc = oracle.encode(v[None], None, NORM_NONE, codec, B=128, s=1, t=t)
+            out = oracle.decode_aggregate(codes, sc, 512, None, NORM_NONE, codec, B=128, s=1)
+            assert np.all(sc == tiny) and not out[v == 0].any()
 
 
 def test_zero_and_nonfinite_blocks_give_zero_codes():
