@@ -1,0 +1,498 @@
+// libtng C ABI: context, workspace, the round of Algorithm 1 as a sequence of
+// kernel launches on one stream (no host synchronisation inside a round).
+#include <math.h>
+#include <stdlib.h>
+#include <string.h>
+
+#include <new>
+
+#include "tng_internal.h"
+
+using namespace tng;
+
+namespace {
+
+constexpr size_t kAlign = 256;
+constexpr int kTimedRounds = 64;   // event sets kept before they are harvested
+constexpr int kStages = 5;         // dots, solve, combine, encode, decode
+
+size_t align_up(size_t x) { return (x + kAlign - 1) / kAlign * kAlign; }
+
+}  // namespace
+
+struct tng_ctx {
+    uint64_t d = 0;
+    uint32_t M = 0, K = 0;
+    int codec = 0, norm = 0;
+    // options
+    uint64_t block_opt = 128;
+    int levels = 7, scale_kind = 0, fuse_mode = TNG_FUSE_AUTO, timing = 0, host_staging = 0;
+    uint32_t seed_lo = 0, seed_hi = 0;
+    double ridge = 1e-6;
+    float quot_eps = 0.0625f;
+    // derived geometry
+    bool sized = false;
+    uint64_t d_pad = 0;
+    CodecGeom geom{};
+    // workspace
+    void* ws = nullptr;
+    size_t ws_bytes = 0;
+    bool ws_owned = false, ws_ready = false;
+    size_t off_ring = 0, off_ref = 0, off_codes = 0, off_scales = 0, off_tile_stat = 0, off_tree = 0,
+           off_partials = 0, off_fb = 0, off_stage_g = 0, off_stage_o = 0;
+    // state
+    uint32_t k = 0;
+    int head = 0;
+    uint64_t rounds = 0;
+    const float* ref_cur = nullptr;   // reference of the last fusion (ref buffer or a ring slot)
+    int last_mode = TNG_FUSE_LAST;
+    bool last_had_stats = false;
+    // bookkeeping
+    int device = 0, sm_count = 148;
+    cudaStream_t last_stream = nullptr;
+    int last_cuda_error = 0;
+    uint64_t launches = 0;
+    unsigned long long nonfinite_reported = 0;
+    // timing
+    cudaEvent_t ev[kTimedRounds][kStages + 1];
+    bool ev_created = false;
+    int ev_used = 0;
+    uint64_t timed_rounds = 0;
+    double ms_sum[kStages] = {0, 0, 0, 0, 0};
+    bool ev_stage_ran[kTimedRounds][kStages];
+
+    float* ring(int slot) const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_ring) + (size_t)slot * d_pad; }
+    float* ref_buf() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_ref); }
+    uint32_t* codes() const { return reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + off_codes); }
+    float* scales() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_scales); }
+    float* tile_stat() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_tile_stat); }
+    float* tree() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_tree); }
+    double* partials() const { return reinterpret_cast<double*>(static_cast<char*>(ws) + off_partials); }
+    FuseBlock* fb() const { return reinterpret_cast<FuseBlock*>(static_cast<char*>(ws) + off_fb); }
+    float* stage_g() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_stage_g); }
+    float* stage_o() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_stage_o); }
+    int hist_slot(uint32_t j) const { return (int)(((int64_t)head - (int64_t)j) % (int64_t)K + (int64_t)K) % (int)K; }
+    int effective_mode() const {
+        if (fuse_mode != TNG_FUSE_AUTO) return fuse_mode;
+        return K == 1 ? TNG_FUSE_LAST : TNG_FUSE_LSQ;
+    }
+};
+
+namespace {
+
+tng_status cuda_fail(tng_ctx* c, cudaError_t e) {
+    if (c) c->last_cuda_error = (int)e;
+    return TNG_ERR_CUDA;
+}
+#define TNG_CUDA(ctx, call)                                  \
+    do {                                                     \
+        cudaError_t e__ = (call);                            \
+        if (e__ != cudaSuccess) return cuda_fail((ctx), e__); \
+    } while (0)
+
+bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Freeze the options into the geometry and the workspace layout.
+void size_ctx(tng_ctx* c) {
+    if (c->sized) return;
+    c->d_pad = (c->d + 31) / 32 * 32;
+    CodecGeom& g = c->geom;
+    g.d = c->d;
+    g.ntile = (c->d + TNG_TILE - 1) / TNG_TILE;
+    g.block = c->block_opt == 0 ? c->d : c->block_opt;
+    g.nblk = c->block_opt == 0 ? 1 : (c->d + c->block_opt - 1) / c->block_opt;
+    g.wpw = g.ntile * 4u * (uint64_t)c->codec;
+    g.M = c->M; g.codec = c->codec; g.norm = c->norm; g.scale_kind = c->scale_kind; g.levels = c->levels;
+    g.seed_lo = c->seed_lo; g.seed_hi = c->seed_hi; g.quot_eps = c->quot_eps;
+    size_t off = 0;
+    c->off_ring = off;      off += align_up((size_t)c->K * c->d_pad * sizeof(float));
+    c->off_ref = off;       off += align_up((size_t)c->d_pad * sizeof(float));
+    c->off_codes = off;     off += align_up((size_t)c->M * g.wpw * sizeof(uint32_t));
+    c->off_scales = off;    off += align_up((size_t)c->M * g.nblk * sizeof(float));
+    const bool general = g.block != TNG_TILE;
+    c->off_tile_stat = off; off += align_up(general ? (size_t)c->M * g.ntile * sizeof(float) : 0);
+    c->off_tree = off;      off += align_up(tree_tmp_floats(g) * sizeof(float));
+    c->off_partials = off;  off += align_up((size_t)kDotsMaxCtas * kDotsMaxAcc * sizeof(double));
+    c->off_fb = off;        off += align_up(sizeof(FuseBlock));
+    c->off_stage_g = off;   off += align_up(c->host_staging ? (size_t)c->M * c->d_pad * sizeof(float) : 0);
+    c->off_stage_o = off;   off += align_up(c->host_staging ? (size_t)c->d_pad * sizeof(float) : 0);
+    c->ws_bytes = off;
+    c->sized = true;
+}
+
+// First device use: pick the device, allocate if nothing was bound, clear the small state block.
+tng_status ensure_ready(tng_ctx* c, cudaStream_t st) {
+    c->last_stream = st;
+    if (c->ws_ready) return TNG_OK;
+    size_ctx(c);
+    TNG_CUDA(c, cudaGetDevice(&c->device));
+    int sms = 0;
+    TNG_CUDA(c, cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, c->device));
+    if (sms > 0) c->sm_count = sms;
+    if (!c->ws) {
+        cudaError_t e = cudaMalloc(&c->ws, c->ws_bytes);
+        if (e != cudaSuccess) {
+            c->last_cuda_error = (int)e;
+            c->ws = nullptr;
+            (void)cudaGetLastError();
+            return TNG_ERR_ALLOC;
+        }
+        c->ws_owned = true;
+    }
+    TNG_CUDA(c, cudaMemsetAsync(c->fb(), 0, sizeof(FuseBlock), st));
+    c->ws_ready = true;
+    return TNG_OK;
+}
+
+tng_status check_rows(const tng_ctx* c, const float* p, uint64_t ld) {
+    if (!p || !aligned16(p) || ld < c->d || (ld % 4) != 0) return TNG_ERR_INVALID_ARG;
+    return TNG_OK;
+}
+
+// ---- timing helpers ---------------------------------------------------------------
+void harvest_events(tng_ctx* c) {
+    if (!c->ev_created || c->ev_used == 0) return;
+    cudaEventSynchronize(c->ev[c->ev_used - 1][kStages]);
+    for (int r = 0; r < c->ev_used; ++r) {
+        for (int s = 0; s < kStages; ++s) {
+            if (!c->ev_stage_ran[r][s]) continue;
+            float ms = 0.f;
+            if (cudaEventElapsedTime(&ms, c->ev[r][s], c->ev[r][s + 1]) == cudaSuccess) c->ms_sum[s] += ms;
+        }
+        c->timed_rounds += 1;
+    }
+    c->ev_used = 0;
+}
+
+struct StageTimer {
+    tng_ctx* c;
+    cudaStream_t st;
+    int slot = -1;
+    StageTimer(tng_ctx* ctx, cudaStream_t s) : c(ctx), st(s) {
+        if (!c->timing) return;
+        if (!c->ev_created) {
+            for (int r = 0; r < kTimedRounds; ++r)
+                for (int s2 = 0; s2 <= kStages; ++s2) cudaEventCreate(&c->ev[r][s2]);
+            c->ev_created = true;
+        }
+        if (c->ev_used == kTimedRounds) harvest_events(c);
+        slot = c->ev_used++;
+        for (int s2 = 0; s2 < kStages; ++s2) c->ev_stage_ran[slot][s2] = false;
+        cudaEventRecord(c->ev[slot][0], st);
+    }
+    // called after stage s has been enqueued; stages must be marked in order 0..4
+    void mark(int s, bool ran) {
+        if (slot < 0) return;
+        c->ev_stage_ran[slot][s] = ran;
+        cudaEventRecord(c->ev[slot][s + 1], st);
+    }
+};
+
+// ---- the stages -----------------------------------------------------------------------
+tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st, StageTimer* tm) {
+    const int mode = c->effective_mode();
+    c->last_mode = mode;
+    c->last_had_stats = false;
+    int launches = 0;
+    if (c->k == 0) {   // empty trajectory: reference = zeros (initial state of Algorithm 1)
+        TNG_CUDA(c, cudaMemsetAsync(c->ref_buf(), 0, c->d_pad * sizeof(float), st));
+        c->ref_cur = c->ref_buf();
+        if (tm) { tm->mark(0, false); tm->mark(1, false); tm->mark(2, false); }
+        return TNG_OK;
+    }
+    const float* rows[kMaxK];
+    for (uint32_t j = 0; j < c->k; ++j) rows[j] = c->ring(c->hist_slot(j));
+    if (mode == TNG_FUSE_LAST) {   // delayed-gradient reference: alias the newest slot, no pass
+        c->ref_cur = rows[0];
+        if (tm) { tm->mark(0, false); tm->mark(1, false); tm->mark(2, false); }
+        return TNG_OK;
+    }
+    const bool need_dots = (mode == TNG_FUSE_LSQ) || (mode == TNG_FUSE_HINDSIGHT);
+    if (need_dots) {
+        const float* g = (mode == TNG_FUSE_LSQ) ? grads : nullptr;
+        TNG_CUDA(c, launch_dots(rows, (int)c->k, c->d, g, c->M, ld, c->partials(), c->fb(), c->sm_count, st, &launches));
+        c->last_had_stats = true;
+    }
+    if (tm) tm->mark(0, need_dots);
+    TNG_CUDA(c, launch_solve(c->fb(), (int)c->k, mode, c->ridge, c->M, st, &launches));
+    if (tm) tm->mark(1, true);
+    TNG_CUDA(c, launch_combine(rows, (int)c->k, c->d, c->fb(), c->ref_buf(), c->sm_count, st, &launches));
+    if (tm) tm->mark(2, true);
+    c->ref_cur = c->ref_buf();
+    c->launches += (uint64_t)launches;
+    return TNG_OK;
+}
+
+tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* ref, uint32_t step, cudaStream_t st) {
+    int launches = 0;
+    TNG_CUDA(c, launch_encode(c->geom, grads, ld, ref, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
+                              c->fb(), c->sm_count, st, &launches));
+    c->launches += (uint64_t)launches;
+    return TNG_OK;
+}
+
+tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, cudaStream_t st) {
+    int launches = 0;
+    TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), ref, out_a, out_b, c->sm_count, st, &launches));
+    c->launches += (uint64_t)launches;
+    return TNG_OK;
+}
+
+tng_status step_impl(tng_ctx* c, const float* grads, uint64_t ld, float* out, cudaStream_t st) {
+    StageTimer tm(c, st);
+    tng_status s = do_fuse(c, grads, ld, st, &tm);
+    if (s != TNG_OK) return s;
+    s = do_encode(c, grads, ld, c->ref_cur, (uint32_t)c->rounds, st);
+    if (s != TNG_OK) return s;
+    tm.mark(3, true);
+    // the decoded aggregate goes straight into the next ring slot (and to the caller's buffer)
+    const int slot = (c->k == 0) ? c->head : (c->head + 1) % (int)c->K;
+    s = do_decode(c, c->ref_cur, c->ring(slot), out, st);
+    if (s != TNG_OK) return s;
+    tm.mark(4, true);
+    c->head = slot;
+    if (c->k < c->K) c->k += 1;
+    c->rounds += 1;
+    return TNG_OK;
+}
+
+}  // namespace
+
+// =========================================================================================
+extern "C" {
+
+tng_status tng_create(tng_ctx** out, uint64_t d, uint32_t M, uint32_t K, tng_codec codec, tng_norm_mode norm) {
+    if (!out) return TNG_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (d < 1 || d > (1ull << 40) || M < 1 || M > TNG_MAX_WORKERS || K < 1 || K > TNG_MAX_HISTORY) return TNG_ERR_INVALID_ARG;
+    if (codec != TNG_CODEC_SIGN1 && codec != TNG_CODEC_TERN2 && codec != TNG_CODEC_QSGD4) return TNG_ERR_INVALID_ARG;
+    if (norm != TNG_NORM_NONE && norm != TNG_NORM_DIFF && norm != TNG_NORM_QUOT) return TNG_ERR_INVALID_ARG;
+    tng_ctx* c = new (std::nothrow) tng_ctx();
+    if (!c) return TNG_ERR_ALLOC;
+    c->d = d; c->M = M; c->K = K; c->codec = (int)codec; c->norm = (int)norm;
+    *out = c;
+    return TNG_OK;
+}
+
+void tng_destroy(tng_ctx* c) {
+    if (!c) return;
+    if (c->ws_ready) cudaStreamSynchronize(c->last_stream);
+    if (c->ev_created)
+        for (int r = 0; r < kTimedRounds; ++r)
+            for (int s = 0; s <= kStages; ++s) cudaEventDestroy(c->ev[r][s]);
+    if (c->ws_owned && c->ws) cudaFree(c->ws);
+    delete c;
+}
+
+tng_status tng_set_option(tng_ctx* c, tng_option key, double value) {
+    if (!c) return TNG_ERR_INVALID_ARG;
+    if (c->sized) return TNG_ERR_STATE;
+    if (!(value == value)) return TNG_ERR_INVALID_ARG;
+    switch (key) {
+        case TNG_OPT_BLOCK:
+            if (value < 0 || value > 1e15 || value != floor(value) || ((uint64_t)value % TNG_TILE) != 0) return TNG_ERR_INVALID_ARG;
+            c->block_opt = (uint64_t)value; return TNG_OK;
+        case TNG_OPT_QSGD_LEVELS:
+            if (value < 1 || value > 7 || value != floor(value)) return TNG_ERR_INVALID_ARG;
+            c->levels = (int)value; return TNG_OK;
+        case TNG_OPT_SCALE_KIND:
+            if (value != 0 && value != 1) return TNG_ERR_INVALID_ARG;
+            c->scale_kind = (int)value; return TNG_OK;
+        case TNG_OPT_SEED_LO:
+        case TNG_OPT_SEED_HI:
+            if (value < 0 || value > 4294967295.0 || value != floor(value)) return TNG_ERR_INVALID_ARG;
+            (key == TNG_OPT_SEED_LO ? c->seed_lo : c->seed_hi) = (uint32_t)value; return TNG_OK;
+        case TNG_OPT_FUSE_MODE:
+            if (value < 0 || value > 4 || value != floor(value)) return TNG_ERR_INVALID_ARG;
+            c->fuse_mode = (int)value; return TNG_OK;
+        case TNG_OPT_RIDGE:
+            if (!(value >= 0) || !(value < 1e300)) return TNG_ERR_INVALID_ARG;
+            c->ridge = value; return TNG_OK;
+        case TNG_OPT_QUOT_EPS:
+            if (!(value > 0 && value <= 1)) return TNG_ERR_INVALID_ARG;
+            c->quot_eps = (float)value; return TNG_OK;
+        case TNG_OPT_TIMING:
+            if (value != 0 && value != 1) return TNG_ERR_INVALID_ARG;
+            c->timing = (int)value; return TNG_OK;
+        case TNG_OPT_HOST_STAGING:
+            if (value != 0 && value != 1) return TNG_ERR_INVALID_ARG;
+            c->host_staging = (int)value; return TNG_OK;
+        default: return TNG_ERR_INVALID_ARG;
+    }
+}
+
+tng_status tng_workspace_bytes(tng_ctx* c, size_t* bytes) {
+    if (!c || !bytes) return TNG_ERR_INVALID_ARG;
+    size_ctx(c);
+    *bytes = c->ws_bytes;
+    return TNG_OK;
+}
+
+tng_status tng_bind_workspace(tng_ctx* c, void* dev_ptr, size_t bytes) {
+    if (!c || !dev_ptr) return TNG_ERR_INVALID_ARG;
+    if (c->ws_ready || c->ws) return TNG_ERR_STATE;
+    if ((reinterpret_cast<uintptr_t>(dev_ptr) % kAlign) != 0) return TNG_ERR_INVALID_ARG;
+    size_ctx(c);
+    if (bytes < c->ws_bytes) return TNG_ERR_ALLOC;
+    c->ws = dev_ptr;
+    c->ws_owned = false;
+    return TNG_OK;
+}
+
+tng_status tng_push_reference(tng_ctx* c, const float* vec_dev, void* stream) {
+    if (!c || !vec_dev || !aligned16(vec_dev)) return TNG_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    const int slot = (c->k == 0) ? c->head : (c->head + 1) % (int)c->K;
+    TNG_CUDA(c, cudaMemcpyAsync(c->ring(slot), vec_dev, c->d * sizeof(float), cudaMemcpyDeviceToDevice, st));
+    c->head = slot;
+    if (c->k < c->K) c->k += 1;
+    return TNG_OK;
+}
+
+tng_status tng_step(tng_ctx* c, const float* grads_dev, uint64_t ld, float* agg_out_dev, void* stream) {
+    if (!c) return TNG_ERR_INVALID_ARG;
+    tng_status s = check_rows(c, grads_dev, ld);
+    if (s != TNG_OK) return s;
+    if (agg_out_dev && !aligned16(agg_out_dev)) return TNG_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    return step_impl(c, grads_dev, ld, agg_out_dev, st);
+}
+
+tng_status tng_step_host(tng_ctx* c, const float* grads_host, uint64_t ld, float* agg_out_host, void* stream) {
+    if (!c || !grads_host || !agg_out_host || ld < c->d) return TNG_ERR_INVALID_ARG;
+    if (!c->host_staging) return TNG_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    TNG_CUDA(c, cudaMemcpy2DAsync(c->stage_g(), c->d_pad * sizeof(float), grads_host, ld * sizeof(float),
+                                  c->d * sizeof(float), c->M, cudaMemcpyHostToDevice, st));
+    s = step_impl(c, c->stage_g(), c->d_pad, c->stage_o(), st);
+    if (s != TNG_OK) return s;
+    TNG_CUDA(c, cudaMemcpyAsync(agg_out_host, c->stage_o(), c->d * sizeof(float), cudaMemcpyDeviceToHost, st));
+    TNG_CUDA(c, cudaStreamSynchronize(st));
+    return TNG_OK;
+}
+
+tng_status tng_fuse(tng_ctx* c, const float* grads_dev, uint64_t ld, void* stream) {
+    if (!c) return TNG_ERR_INVALID_ARG;
+    tng_status s = check_rows(c, grads_dev, ld);
+    if (s != TNG_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    return do_fuse(c, grads_dev, ld, st, nullptr);
+}
+
+tng_status tng_encode(tng_ctx* c, const float* grads_dev, uint64_t ld, const float* ref_dev, uint32_t step, void* stream) {
+    if (!c) return TNG_ERR_INVALID_ARG;
+    tng_status s = check_rows(c, grads_dev, ld);
+    if (s != TNG_OK) return s;
+    if (ref_dev && !aligned16(ref_dev)) return TNG_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    const float* ref = ref_dev ? ref_dev : c->ref_cur;
+    if (!ref && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;   // no fusion has produced a reference yet
+    return do_encode(c, grads_dev, ld, ref, step, st);
+}
+
+tng_status tng_decode_aggregate(tng_ctx* c, const float* ref_dev, float* out_dev, void* stream) {
+    if (!c || !out_dev || !aligned16(out_dev)) return TNG_ERR_INVALID_ARG;
+    if (ref_dev && !aligned16(ref_dev)) return TNG_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    const float* ref = ref_dev ? ref_dev : c->ref_cur;
+    if (!ref && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;
+    return do_decode(c, ref, out_dev, nullptr, st);
+}
+
+tng_status tng_wire(tng_ctx* c, const uint32_t** codes_dev, size_t* words_per_worker, const float** scales_dev,
+                    size_t* scales_per_worker) {
+    if (!c) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready) return TNG_ERR_STATE;
+    if (codes_dev) *codes_dev = c->codes();
+    if (words_per_worker) *words_per_worker = (size_t)c->geom.wpw;
+    if (scales_dev) *scales_dev = c->scales();
+    if (scales_per_worker) *scales_per_worker = (size_t)c->geom.nblk;
+    return TNG_OK;
+}
+
+tng_status tng_reference(tng_ctx* c, const float** ref_dev) {
+    if (!c || !ref_dev) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready || !c->ref_cur) return TNG_ERR_STATE;
+    *ref_dev = c->ref_cur;
+    return TNG_OK;
+}
+
+tng_status tng_history(tng_ctx* c, uint32_t j, const float** vec_dev) {
+    if (!c || !vec_dev) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready || j >= c->k) return TNG_ERR_STATE;
+    *vec_dev = c->ring(c->hist_slot(j));
+    return TNG_OK;
+}
+
+tng_status tng_stats(tng_ctx* c, tng_stats_t* out) {
+    if (!c || !out) return TNG_ERR_INVALID_ARG;
+    memset(out, 0, sizeof *out);
+    size_ctx(c);
+    out->d = c->d; out->M = c->M; out->K = c->K; out->k = c->k;
+    out->fuse_mode = (uint32_t)c->effective_mode();
+    out->rounds = c->rounds;
+    out->bits_per_coord = (double)c->codec + 32.0 / (double)c->geom.block + 64.0 * (double)c->K / (double)c->d;
+    out->cnz = nan("");
+    out->kernel_launches = c->launches;
+    if (!c->ws_ready) return TNG_OK;
+    TNG_CUDA(c, cudaStreamSynchronize(c->last_stream));
+    harvest_events(c);
+    FuseBlock h;
+    TNG_CUDA(c, cudaMemcpy(&h, c->fb(), sizeof h, cudaMemcpyDeviceToHost));
+    const int mode = c->last_mode;
+    if (mode == TNG_FUSE_LAST || c->rounds == 0) {
+        out->alpha[0] = (c->k > 0 || c->rounds > 0) ? 1.0 : 0.0;
+    } else {
+        for (int j = 0; j < TNG_MAX_HISTORY; ++j) out->alpha[j] = h.alpha64[j];
+        out->solver_fallback = h.fallback;
+    }
+    if (c->last_had_stats) {
+        for (int i = 0; i < TNG_MAX_HISTORY * TNG_MAX_HISTORY; ++i) out->gram[i] = h.gram[i];
+        if (mode == TNG_FUSE_LSQ) {
+            for (int i = 0; i < TNG_MAX_HISTORY; ++i) out->rhs[i] = h.gram[kGramRhs + i];
+            out->grad_sq = h.gram[kGramGG];
+            out->cnz = h.cnz;
+        }
+    }
+    out->nonfinite_scales = h.nonfinite;
+    out->timed_rounds = c->timed_rounds;
+    if (c->timed_rounds) {
+        const double n = (double)c->timed_rounds;
+        out->ms_dots = c->ms_sum[0] / n; out->ms_solve = c->ms_sum[1] / n; out->ms_combine = c->ms_sum[2] / n;
+        out->ms_encode = c->ms_sum[3] / n; out->ms_decode = c->ms_sum[4] / n;
+    }
+    if (h.nonfinite > c->nonfinite_reported) {
+        c->nonfinite_reported = h.nonfinite;
+        return TNG_ERR_NONFINITE;
+    }
+    return TNG_OK;
+}
+
+const char* tng_status_string(tng_status s) {
+    switch (s) {
+        case TNG_OK: return "ok";
+        case TNG_ERR_INVALID_ARG: return "invalid argument";
+        case TNG_ERR_STATE: return "call not allowed in this state";
+        case TNG_ERR_ALLOC: return "allocation failed or workspace too small";
+        case TNG_ERR_CUDA: return "CUDA error";
+        case TNG_ERR_NONFINITE: return "non-finite block scale";
+        case TNG_ERR_UNSUPPORTED: return "unsupported";
+        default: return "unknown status";
+    }
+}
+
+int tng_last_cuda_error(const tng_ctx* c) { return c ? c->last_cuda_error : 0; }
+
+}  // extern "C"

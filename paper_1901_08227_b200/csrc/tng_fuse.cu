@@ -1,0 +1,397 @@
+// Trajectory fusion kernels (sm_100a): the sufficient statistics of
+//   min_alpha sum_m || g^m - sum_j alpha_j h_j ||^2
+// (the C_nz criterion of Proposition 2 over the span of the stored aggregates of
+// Section 3.1): Gram G = <h_i,h_j>, rhs c_i = <h_i, mean gradient>; a K x K
+// ridge solve; and the reference combine r = sum_j alpha_j h_j.
+//
+// The statistics pass is one streaming sweep over the ring and the M gradient
+// rows.  Each thread owns four coordinates per iteration (128-bit loads of all
+// k + M vectors), converts them to double once and accumulates every pair
+// product in double, so the result does not depend on how the sum is split.
+// Per-CTA partials are combined in CTA order by the CTA that finishes last
+// (an arrival counter, nobody waits), which keeps the sums run-to-run identical.
+#include "tng_device.cuh"
+#include "tng_internal.h"
+
+namespace tng {
+
+namespace {
+
+constexpr int kDotsThreads = 256;
+
+struct DotsArgs {
+    const float* rows_a[8];
+    const float* rows_b[8];
+    const float* grads;       // nullptr: Gram only
+    double* partials;         // gridDim.x * kDotsMaxAcc
+    FuseBlock* fb;
+    uint64_t d, ld;
+    uint32_t M;
+    short dst[kDotsMaxAcc];   // destination of accumulator i inside fb->gram
+};
+
+template <int NA, int NB, bool SAME>
+struct DotsShape {
+    static constexpr int kPairs = SAME ? NA * (NA + 1) / 2 : NA * NB;
+    static constexpr int kAcc = SAME ? kPairs + NA + 1 : kPairs;   // + rhs + grad_sq
+};
+
+template <int NA, int NB, bool SAME>
+__global__ void __launch_bounds__(kDotsThreads, 1) dots_kernel(const DotsArgs a) {
+    using Shape = DotsShape<NA, NB, SAME>;
+    constexpr int kAcc = Shape::kAcc;
+    double acc[kAcc];
+#pragma unroll
+    for (int i = 0; i < kAcc; ++i) acc[i] = 0.0;
+    const bool with_g = SAME && (a.grads != nullptr);
+
+    const uint64_t ngroups = (a.d + 3) / 4;
+    const uint64_t stride = (uint64_t)gridDim.x * kDotsThreads;
+    for (uint64_t grp = (uint64_t)blockIdx.x * kDotsThreads + threadIdx.x; grp < ngroups; grp += stride) {
+        const uint64_t i0 = grp * 4;
+        float4 ha[NA];
+        float4 hb[SAME ? 1 : NB];
+#pragma unroll
+        for (int j = 0; j < NA; ++j) ha[j] = load4_stream(a.rows_a[j], i0, a.d);
+        if (!SAME) {
+#pragma unroll
+            for (int j = 0; j < NB; ++j) hb[j] = load4_stream(a.rows_b[j], i0, a.d);
+        }
+        // sum and sum of squares of the M gradients at these coordinates (fp32, m ascending)
+        float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), gq = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (with_g) {
+            for (uint32_t m0 = 0; m0 < a.M; m0 += 8) {
+                float4 g[8];
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (m0 + k < a.M) g[k] = load4_stream(a.grads + (uint64_t)(m0 + k) * a.ld, i0, a.d);
+#pragma unroll
+                for (int k = 0; k < 8; ++k)
+                    if (m0 + k < a.M) {
+                        gs.x += g[k].x; gs.y += g[k].y; gs.z += g[k].z; gs.w += g[k].w;
+                        gq.x = fmaf(g[k].x, g[k].x, gq.x); gq.y = fmaf(g[k].y, g[k].y, gq.y);
+                        gq.z = fmaf(g[k].z, g[k].z, gq.z); gq.w = fmaf(g[k].w, g[k].w, gq.w);
+                    }
+            }
+        }
+#pragma unroll
+        for (int comp = 0; comp < 4; ++comp) {
+            double da[NA];
+#pragma unroll
+            for (int j = 0; j < NA; ++j) da[j] = (double)(comp == 0 ? ha[j].x : comp == 1 ? ha[j].y : comp == 2 ? ha[j].z : ha[j].w);
+            if (SAME) {
+                int p = 0;
+#pragma unroll
+                for (int i = 0; i < NA; ++i)
+#pragma unroll
+                    for (int j = i; j < NA; ++j) { acc[p] = fma(da[i], da[j], acc[p]); ++p; }
+                if (with_g) {
+                    const double dg = (double)(comp == 0 ? gs.x : comp == 1 ? gs.y : comp == 2 ? gs.z : gs.w);
+#pragma unroll
+                    for (int i = 0; i < NA; ++i) acc[Shape::kPairs + i] = fma(da[i], dg, acc[Shape::kPairs + i]);
+                    acc[Shape::kPairs + NA] += (double)(comp == 0 ? gq.x : comp == 1 ? gq.y : comp == 2 ? gq.z : gq.w);
+                }
+            } else {
+                double db[SAME ? 1 : NB];
+#pragma unroll
+                for (int j = 0; j < NB; ++j) db[j] = (double)(comp == 0 ? hb[j].x : comp == 1 ? hb[j].y : comp == 2 ? hb[j].z : hb[j].w);
+#pragma unroll
+                for (int i = 0; i < NA; ++i)
+#pragma unroll
+                    for (int j = 0; j < NB; ++j) acc[i * NB + j] = fma(da[i], db[j], acc[i * NB + j]);
+            }
+        }
+    }
+
+    // ---- CTA reduction: lanes by butterfly, warps in warp order
+    __shared__ double warp_part[kDotsThreads / 32][kAcc];
+    __shared__ bool is_last;
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int i = 0; i < kAcc; ++i) {
+        double v = acc[i];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(kFullMask, v, off);
+        if (lane == 0) warp_part[warp][i] = v;
+    }
+    __syncthreads();
+    if (threadIdx.x < kAcc) {
+        double v = 0.0;
+        for (int w = 0; w < kDotsThreads / 32; ++w) v += warp_part[w][threadIdx.x];
+        a.partials[(uint64_t)blockIdx.x * kDotsMaxAcc + threadIdx.x] = v;
+    }
+    // ---- the CTA that arrives last adds the partials in CTA order
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const uint32_t prev = atomicAdd(&a.fb->dots_arrivals, 1u);
+        is_last = (prev == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    if (threadIdx.x < kAcc) {
+        double v = 0.0;
+        for (uint32_t b = 0; b < gridDim.x; ++b) v += __ldcg(a.partials + (uint64_t)b * kDotsMaxAcc + threadIdx.x);
+        if (SAME && threadIdx.x >= Shape::kPairs) v /= (double)a.M;   // rhs and grad_sq use the mean
+        if (!(SAME && !with_g && threadIdx.x >= Shape::kPairs)) a.fb->gram[a.dst[threadIdx.x]] = v;
+    }
+    if (threadIdx.x == 0) a.fb->dots_arrivals = 0;   // ready for the next launch on this stream
+}
+
+template <int NA>
+cudaError_t dots_same(const DotsArgs& a, int grid, cudaStream_t st) {
+    dots_kernel<NA, NA, true><<<grid, kDotsThreads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template <int NB>
+cudaError_t dots_cross(const DotsArgs& a, int grid, cudaStream_t st) {
+    dots_kernel<8, NB, false><<<grid, kDotsThreads, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+cudaError_t dots_same_n(int n, const DotsArgs& a, int grid, cudaStream_t st) {
+    switch (n) {
+        case 1: return dots_same<1>(a, grid, st);
+        case 2: return dots_same<2>(a, grid, st);
+        case 3: return dots_same<3>(a, grid, st);
+        case 4: return dots_same<4>(a, grid, st);
+        case 5: return dots_same<5>(a, grid, st);
+        case 6: return dots_same<6>(a, grid, st);
+        case 7: return dots_same<7>(a, grid, st);
+        default: return dots_same<8>(a, grid, st);
+    }
+}
+cudaError_t dots_cross_n(int n, const DotsArgs& a, int grid, cudaStream_t st) {
+    switch (n) {
+        case 1: return dots_cross<1>(a, grid, st);
+        case 2: return dots_cross<2>(a, grid, st);
+        case 3: return dots_cross<3>(a, grid, st);
+        case 4: return dots_cross<4>(a, grid, st);
+        case 5: return dots_cross<5>(a, grid, st);
+        case 6: return dots_cross<6>(a, grid, st);
+        case 7: return dots_cross<7>(a, grid, st);
+        default: return dots_cross<8>(a, grid, st);
+    }
+}
+
+// ---------------------------------------------------------------------------
+// K x K solve: one warp, lane 0 runs the Cholesky in double (k <= 16).
+// mode: TNG_FUSE_LSQ, TNG_FUSE_HINDSIGHT, TNG_FUSE_MEAN.
+// ---------------------------------------------------------------------------
+__device__ bool chol_solve(const double* A, const double* rhs, int n, double* x) {
+    double L[kMaxK * kMaxK];
+    double y[kMaxK];
+    for (int j = 0; j < n; ++j) {
+        double diag = A[j * n + j];
+        for (int p = 0; p < j; ++p) diag -= L[j * n + p] * L[j * n + p];
+        // a pivot that is not above 1e-12 of its diagonal entry is rounding noise of a singular matrix
+        if (!(diag > 1e-12 * A[j * n + j]) || !(diag > 0.0) || !isfinite(diag)) return false;
+        const double ljj = sqrt(diag);
+        L[j * n + j] = ljj;
+        for (int i = j + 1; i < n; ++i) {
+            double v = A[i * n + j];
+            for (int p = 0; p < j; ++p) v -= L[i * n + p] * L[j * n + p];
+            L[i * n + j] = v / ljj;
+        }
+    }
+    for (int i = 0; i < n; ++i) {
+        double v = rhs[i];
+        for (int p = 0; p < i; ++p) v -= L[i * n + p] * y[p];
+        y[i] = v / L[i * n + i];
+    }
+    for (int i = n - 1; i >= 0; --i) {
+        double v = y[i];
+        for (int p = i + 1; p < n; ++p) v -= L[p * n + i] * x[p];
+        x[i] = v / L[i * n + i];
+    }
+    for (int i = 0; i < n; ++i)
+        if (!isfinite(x[i])) return false;
+    return true;
+}
+
+__global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mode, double ridge, int have_rhs) {
+    if (threadIdx.x != 0) return;
+    double alpha[kMaxK];
+    for (int j = 0; j < kMaxK; ++j) alpha[j] = 0.0;
+    uint32_t fallback = 0;
+    double* G = fb->gram;
+    if (mode == TNG_FUSE_MEAN) {
+        const float inv = __fdiv_rn(1.0f, (float)k);
+        for (int j = 0; j < k; ++j) alpha[j] = (double)inv;
+    } else {
+        for (int a = 0; a < k; ++a)   // mirror the upper triangle
+            for (int b = 0; b < a; ++b) G[a * kGramStride + b] = G[b * kGramStride + a];
+        double A[kMaxK * kMaxK], rhs[kMaxK], x[kMaxK];
+        bool ok;
+        if (mode == TNG_FUSE_LSQ) {
+            double trace = 0.0;
+            for (int j = 0; j < k; ++j) trace += G[j * kGramStride + j];
+            const double lambda = ridge * trace / (double)k;
+            for (int a = 0; a < k; ++a) {
+                rhs[a] = G[kGramRhs + a];
+                for (int b = 0; b < k; ++b) A[a * k + b] = G[a * kGramStride + b] + (a == b ? lambda : 0.0);
+            }
+            ok = chol_solve(A, rhs, k, x);
+            if (ok) for (int j = 0; j < k; ++j) alpha[j] = x[j];
+        } else {   // hindsight: regress h_1 on h_2..h_k, apply one position later
+            const int n = k - 1;
+            ok = true;
+            if (n >= 1) {
+                double trace = 0.0;
+                for (int j = 1; j < k; ++j) trace += G[j * kGramStride + j];
+                const double lambda = ridge * trace / (double)n;
+                for (int a = 0; a < n; ++a) {
+                    rhs[a] = G[(a + 1) * kGramStride + 0];
+                    for (int b = 0; b < n; ++b)
+                        A[a * n + b] = G[(a + 1) * kGramStride + (b + 1)] + (a == b ? lambda : 0.0);
+                }
+                ok = chol_solve(A, rhs, n, x);
+                if (ok) for (int j = 0; j < n; ++j) alpha[j] = x[j];
+            } else {
+                alpha[0] = 1.0;
+            }
+        }
+        if (!ok) {
+            fallback = 1;
+            for (int j = 0; j < kMaxK; ++j) alpha[j] = 0.0;
+            alpha[0] = 1.0;
+        }
+    }
+    double a32[kMaxK];
+    for (int j = 0; j < kMaxK; ++j) {
+        fb->alpha64[j] = alpha[j];
+        const float f = (float)alpha[j];
+        fb->alpha32[j] = f;
+        a32[j] = (double)f;
+    }
+    fb->fallback = fallback;
+    // C_nz estimate from the statistics: (gg - 2 a.c + a^T G a) / gg with the fp32 coefficients
+    double cnz = nan("");
+    if (have_rhs && mode != TNG_FUSE_MEAN) {
+        double quad = 0.0, lin = 0.0;
+        for (int a = 0; a < k; ++a) {
+            lin += a32[a] * G[kGramRhs + a];
+            for (int b = 0; b < k; ++b) quad += a32[a] * a32[b] * G[a * kGramStride + b];
+        }
+        const double gg = G[kGramGG];
+        cnz = (gg - 2.0 * lin + quad) / gg;
+    }
+    fb->cnz = cnz;
+}
+
+// ---------------------------------------------------------------------------
+// reference combine: r_d = fma(alpha_k, h_k[d], ... fma(alpha_1, h_1[d], 0)), fp32
+// ---------------------------------------------------------------------------
+struct CombineArgs {
+    const float* rows[kMaxK];
+    const float* alpha;
+    float* ref;
+    uint64_t d;
+};
+
+template <int KK>
+__global__ void __launch_bounds__(256) combine_kernel(const CombineArgs a) {
+    float al[KK];
+#pragma unroll
+    for (int j = 0; j < KK; ++j) al[j] = __ldg(a.alpha + j);
+    const uint64_t ngroups = (a.d + 3) / 4;
+    const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
+    for (uint64_t grp = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x; grp < ngroups; grp += stride) {
+        const uint64_t i0 = grp * 4;
+        float4 h[KK];
+#pragma unroll
+        for (int j = 0; j < KK; ++j) h[j] = load4_stream(a.rows[j], i0, a.d);
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < KK; ++j) {
+            r.x = __fmaf_rn(al[j], h[j].x, r.x); r.y = __fmaf_rn(al[j], h[j].y, r.y);
+            r.z = __fmaf_rn(al[j], h[j].z, r.z); r.w = __fmaf_rn(al[j], h[j].w, r.w);
+        }
+        store4(a.ref, i0, a.d, r);
+    }
+}
+
+template <int KK>
+cudaError_t combine_k(const CombineArgs& a, int grid, cudaStream_t st) {
+    combine_kernel<KK><<<grid, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float* grads, uint32_t M, uint64_t ld,
+                        double* partials, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
+    const uint64_t ngroups = (d + 3) / 4;
+    uint64_t want = (ngroups + kDotsThreads - 1) / kDotsThreads;
+    if (want < 1) want = 1;
+    const int grid = (int)(want < (uint64_t)sm_count ? want : (uint64_t)sm_count);
+    DotsArgs a;
+    a.grads = grads; a.partials = partials; a.fb = fb; a.d = d; a.ld = ld; a.M = M;
+    cudaError_t e = cudaSuccess;
+    // chunks of at most 8 history vectors: diagonal blocks (with rhs) and, for k > 8, the cross block
+    for (int lo = 0; lo < k && e == cudaSuccess; lo += 8) {
+        const int n = (k - lo < 8) ? k - lo : 8;
+        for (int j = 0; j < 8; ++j) a.rows_a[j] = a.rows_b[j] = rows[lo + (j < n ? j : 0)];
+        int p = 0;
+        for (int i = 0; i < n; ++i)
+            for (int j = i; j < n; ++j) a.dst[p++] = (short)((lo + i) * kGramStride + lo + j);
+        for (int i = 0; i < n; ++i) a.dst[p++] = (short)(kGramRhs + lo + i);
+        a.dst[p++] = (short)kGramGG;
+        e = dots_same_n(n, a, grid, st);
+        ++*launches;
+    }
+    if (k > 8 && e == cudaSuccess) {
+        const int nb = k - 8;
+        for (int j = 0; j < 8; ++j) {
+            a.rows_a[j] = rows[j];
+            a.rows_b[j] = rows[8 + (j < nb ? j : 0)];
+        }
+        for (int i = 0; i < 8; ++i)
+            for (int j = 0; j < nb; ++j) a.dst[i * nb + j] = (short)(i * kGramStride + 8 + j);
+        e = dots_cross_n(nb, a, grid, st);
+        ++*launches;
+    }
+    return e;
+}
+
+cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, uint32_t M, cudaStream_t st, int* launches) {
+    (void)M;
+    solve_kernel<<<1, 32, 0, st>>>(fb, k, mode, ridge, mode == TNG_FUSE_LSQ ? 1 : 0);
+    ++*launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const FuseBlock* fb, float* ref, int sm_count,
+                           cudaStream_t st, int* launches) {
+    CombineArgs a;
+    for (int j = 0; j < kMaxK; ++j) a.rows[j] = rows[j < k ? j : 0];
+    a.alpha = fb->alpha32; a.ref = ref; a.d = d;
+    const uint64_t ngroups = (d + 3) / 4;
+    uint64_t want = (ngroups + 255) / 256;
+    const uint64_t cap = (uint64_t)sm_count * 8;
+    const int grid = (int)(want < cap ? (want ? want : 1) : cap);
+    cudaError_t e;
+    switch (k) {
+        case 1: e = combine_k<1>(a, grid, st); break;
+        case 2: e = combine_k<2>(a, grid, st); break;
+        case 3: e = combine_k<3>(a, grid, st); break;
+        case 4: e = combine_k<4>(a, grid, st); break;
+        case 5: e = combine_k<5>(a, grid, st); break;
+        case 6: e = combine_k<6>(a, grid, st); break;
+        case 7: e = combine_k<7>(a, grid, st); break;
+        case 8: e = combine_k<8>(a, grid, st); break;
+        case 9: e = combine_k<9>(a, grid, st); break;
+        case 10: e = combine_k<10>(a, grid, st); break;
+        case 11: e = combine_k<11>(a, grid, st); break;
+        case 12: e = combine_k<12>(a, grid, st); break;
+        case 13: e = combine_k<13>(a, grid, st); break;
+        case 14: e = combine_k<14>(a, grid, st); break;
+        case 15: e = combine_k<15>(a, grid, st); break;
+        default: e = combine_k<16>(a, grid, st); break;
+    }
+    ++*launches;
+    return e;
+}
+
+}  // namespace tng

@@ -1,0 +1,63 @@
+// Host-side declarations shared by the libtng translation units.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "tng.h"
+
+namespace tng {
+
+constexpr int kMaxK = TNG_MAX_HISTORY;
+constexpr int kGramStride = kMaxK;                      // G[a*16 + b]
+constexpr int kGramRhs = kMaxK * kMaxK;                 // c[a] at 256 + a
+constexpr int kGramGG = kGramRhs + kMaxK;               // gg at 272
+constexpr int kGramDoubles = kGramGG + 1;
+constexpr int kDotsMaxAcc = 64;                         // accumulators of one dots launch
+constexpr int kDotsMaxCtas = 592;                       // 4 x 148
+
+// Small device-resident block: fusion statistics, coefficients, flags.
+struct FuseBlock {
+    double gram[kGramDoubles + 7];   // padded to 280 doubles
+    double alpha64[kMaxK];
+    double cnz;
+    float alpha32[kMaxK];
+    uint32_t fallback;
+    uint32_t dots_arrivals;          // CTAs that finished the current dots launch
+    unsigned long long nonfinite;    // NaN/Inf block scales seen so far
+};
+
+struct CodecGeom {
+    uint64_t d;
+    uint64_t ntile;      // ceil(d/128)
+    uint64_t nblk;       // scales per worker
+    uint64_t block;      // coordinates per scale (d for per-vector)
+    uint64_t wpw;        // code words per worker
+    uint32_t M;
+    int codec, norm, scale_kind, levels;
+    uint32_t seed_lo, seed_hi;
+    float quot_eps;
+};
+
+// ---- fusion (tng_fuse.cu) ---------------------------------------------------
+// rows[j] = h_{j+1}.  Accumulates G (and with grads != nullptr the rhs and grad_sq)
+// into fb->gram via per-CTA partials in `partials` (kDotsMaxCtas * kDotsMaxAcc doubles).
+cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float* grads, uint32_t M,
+                        uint64_t ld, double* partials, FuseBlock* fb, int sm_count, cudaStream_t st,
+                        int* launches);
+cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, uint32_t M, cudaStream_t st,
+                         int* launches);
+cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const FuseBlock* fb, float* ref,
+                           int sm_count, cudaStream_t st, int* launches);
+
+// ---- codec (tng_codec.cu) -----------------------------------------------------
+// tile_stat: M*ntile floats, tree_tmp: scratch of tree_tmp_floats(geom) floats; both
+// only used when geom.block != 128.
+size_t tree_tmp_floats(const CodecGeom& g);
+cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref,
+                          uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp,
+                          FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
+cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref,
+                          float* out_a, float* out_b, int sm_count, cudaStream_t st, int* launches);
+
+}  // namespace tng

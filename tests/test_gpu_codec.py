@@ -1,0 +1,157 @@
+"""GPU parity, stage level: tng_encode / tng_decode_aggregate through the C ABI
+against the CPU oracle on the same seeded inputs and the same reference.
+Packed codes, scales and decoded aggregates must match bit for bit."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import codes_np, make_ctx, same_values, to_np
+from paper_1901_08227_b200 import tng, workloads
+
+pytestmark = pytest.mark.gpu
+
+CODECS = [tng.CODEC_SIGN1, tng.CODEC_TERN2, tng.CODEC_QSGD4]
+NORMS = [tng.NORM_NONE, tng.NORM_DIFF, tng.NORM_QUOT]
+
+
+def run_both(d, M, codec, norm, B, scale_kind=0, s=7, seed=(3, 9), step=5, ld=None, kind="normal", ref_kind="near"):
+    dev = "cuda"
+    g = workloads.random_grads(d * 7 + M, M, d, device=dev, ld=ld, kind=kind)
+    if ref_kind == "near":
+        ref = (g.mean(0) * 0.9 + 0.05 * workloads.normal((d,), 11, 1, dev)).contiguous()
+    elif ref_kind == "zeros":
+        ref = torch.zeros(d, device=dev)
+    else:   # sparse: whole tiles of zeros and tiny entries, exercises the quotient guard
+        ref = g.mean(0).clone()
+        ref[: min(d, 200)] = 0.0
+        ref[::7] *= 1e-6
+        ref = ref.contiguous()
+    ctx = make_ctx(d, M, 1, codec, norm, block=B, scale_kind=scale_kind, qsgd_levels=s, seed_lo=seed[0], seed_hi=seed[1])
+    ctx.encode(g, ref=ref if norm != tng.NORM_NONE else None, step=step)
+    codes, scales = ctx.wire()
+    out = torch.empty(d, device=dev)
+    ctx.decode_aggregate(out, ref=ref if norm != tng.NORM_NONE else None)
+    torch.cuda.synchronize()
+    st = ctx.stats()
+    gn, rn = to_np(g), to_np(ref)
+    oc, osc = oracle.encode(gn, rn if norm != tng.NORM_NONE else None, norm, codec, B=B, s=s, scale_kind=scale_kind,
+                            seed=seed, t=step)
+    oout = oracle.decode_aggregate(oc, osc, d, rn if norm != tng.NORM_NONE else None, norm, codec, B=B, s=s)
+    ctx.close()
+    return (codes_np(codes), to_np(scales), to_np(out)), (oc, osc, oout), st
+
+
+def assert_exact(got, want):
+    assert same_values(got[1], want[1]), "scales differ"
+    assert np.array_equal(got[0], want[0]), "packed codes differ"
+    assert same_values(got[2], want[2]), "decoded aggregate differs"
+
+
+@pytest.mark.parametrize("codec", CODECS)
+@pytest.mark.parametrize("norm", NORMS)
+@pytest.mark.parametrize("d,M", [(1, 1), (3, 2), (127, 3), (128, 1), (1000, 4), (4099, 8), (128 * 41, 5)])
+def test_block128_bit_exact(codec, norm, d, M):
+    got, want, _ = run_both(d, M, codec, norm, 128)
+    assert_exact(got, want)
+
+
+@pytest.mark.parametrize("codec", CODECS)
+@pytest.mark.parametrize("scale_kind", [0, 1])
+@pytest.mark.parametrize("B,d", [(0, 1000), (0, 5), (256, 65536 // 8 + 77), (384, 3000), (1024, 128 * 50 + 1), (0, 128 * 2100 + 9)])
+def test_general_block_sizes_bit_exact(codec, scale_kind, B, d):
+    got, want, _ = run_both(d, 3, codec, tng.NORM_DIFF, B, scale_kind=scale_kind, s=4)
+    assert_exact(got, want)
+
+
+@pytest.mark.parametrize("codec", CODECS)
+@pytest.mark.parametrize("norm", [tng.NORM_DIFF, tng.NORM_QUOT])
+def test_l2_scale_block128(codec, norm):
+    got, want, _ = run_both(5000, 4, codec, norm, 128, scale_kind=1)
+    assert_exact(got, want)
+
+
+@pytest.mark.parametrize("s", [1, 2, 3, 4, 5, 6, 7])
+def test_qsgd_levels(s):
+    got, want, _ = run_both(3001, 4, tng.CODEC_QSGD4, tng.NORM_DIFF, 128, s=s)
+    assert_exact(got, want)
+
+
+@pytest.mark.parametrize("norm", [tng.NORM_DIFF, tng.NORM_QUOT])
+@pytest.mark.parametrize("ref_kind", ["zeros", "sparse"])
+def test_degenerate_references(norm, ref_kind):
+    got, want, _ = run_both(2000, 4, tng.CODEC_TERN2, norm, 128, ref_kind=ref_kind)
+    assert_exact(got, want)
+
+
+def test_heavy_tails_row_stride_and_many_workers():
+    got, want, _ = run_both(128 * 64 + 40, 64, tng.CODEC_TERN2, tng.NORM_QUOT, 128, ld=128 * 64 + 44, kind="heavy")
+    assert_exact(got, want)
+    got, want, _ = run_both(10007, 13, tng.CODEC_SIGN1, tng.NORM_DIFF, 128, ld=10008, kind="heavy")
+    assert_exact(got, want)
+
+
+def test_several_tiles_per_warp_and_seeds():
+    # more tiles than resident warps, so every warp loops; several seeds / steps
+    d = 128 * 20000 + 17
+    for seed, step in [((0, 0), 0), ((0xFFFFFFFF, 7), 123456)]:
+        got, want, _ = run_both(d, 2, tng.CODEC_TERN2, tng.NORM_DIFF, 128, seed=seed, step=step)
+        assert_exact(got, want)
+
+
+def test_gradient_equal_to_reference_gives_zero_codes_on_the_gpu():
+    d, M = 1500, 3
+    r = workloads.normal((d,), 5, 0, "cuda")
+    g = r.unsqueeze(0).repeat(M, 1).contiguous()
+    ctx = make_ctx(d, M, 1, tng.CODEC_TERN2, tng.NORM_DIFF)
+    ctx.encode(g, ref=r, step=0)
+    codes, scales = ctx.wire()
+    out = torch.empty(d, device="cuda")
+    ctx.decode_aggregate(out, ref=r)
+    assert not codes.any() and not scales.any()
+    assert torch.equal(out, r)
+
+
+def test_nonfinite_scales_are_counted_and_zeroed():
+    d, M = 1000, 2
+    g = workloads.random_grads(1, M, d, device="cuda")
+    g[0, 300] = float("nan")
+    g[1, 700] = float("inf")
+    ctx = make_ctx(d, M, 1, tng.CODEC_TERN2, tng.NORM_NONE)
+    ctx.encode(g, step=0)
+    codes, scales = ctx.wire()
+    out = torch.empty(d, device="cuda")
+    ctx.decode_aggregate(out)
+    gn = to_np(g)
+    oc, osc = oracle.encode(gn, None, tng.NORM_NONE, tng.CODEC_TERN2, B=128)
+    assert np.array_equal(codes_np(codes), oc) and same_values(to_np(scales), osc)
+    assert same_values(to_np(out), oracle.decode_aggregate(oc, osc, d, None, tng.NORM_NONE, tng.CODEC_TERN2, B=128))
+    with pytest.raises(tng.TngError) as e:
+        ctx.stats(raise_on_nonfinite=True)
+    assert e.value.status == tng.ERR_NONFINITE
+    assert ctx.stats().nonfinite_scales == 2
+    # general block path counts too
+    ctx2 = make_ctx(d, M, 1, tng.CODEC_TERN2, tng.NORM_NONE, block=256)
+    ctx2.encode(g, step=0)
+    assert ctx2.stats().nonfinite_scales == 2
+
+
+def test_argument_checks_return_status_codes():
+    ctx = make_ctx(1000, 2, 1, tng.CODEC_TERN2, tng.NORM_DIFF)
+    g = workloads.random_grads(1, 2, 1000, device="cuda")
+    buf = torch.zeros(2 * 1002 + 8, device="cuda")
+    bad_ld = buf[: 2 * 1002].view(2, 1002)[:, :1000]           # ld = 1002 is not a multiple of 4
+    with pytest.raises(tng.TngError) as e:
+        ctx.step(bad_ld)
+    assert e.value.status == tng.ERR_INVALID_ARG
+    misaligned = buf[1: 1 + 2000].view(2, 1000)                # base not 16-byte aligned
+    with pytest.raises(tng.TngError) as e:
+        ctx.step(misaligned)
+    assert e.value.status == tng.ERR_INVALID_ARG
+    with pytest.raises(tng.TngError) as e:
+        ctx.step_host(torch.zeros(2, 1000), torch.zeros(1000))  # staging was not requested
+    assert e.value.status == tng.ERR_STATE
+    out = torch.empty(1000, device="cuda")
+    ctx.step(g, out)                                            # still usable afterwards
+    torch.cuda.synchronize()
+    assert torch.isfinite(out).all()
