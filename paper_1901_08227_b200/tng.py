@@ -86,10 +86,6 @@ def lib():
         L.tng_rosenbrock_grad.argtypes = [vp, u64, vp, u32, u64, vp, vp]
         L.tng_rosenbrock_value.argtypes = [vp, u64, vp, vp]
         L.tng_sgd_update.argtypes = [vp, vp, u64, f32, vp]
-        if hasattr(L, "tng_gram_static"):
-            L.tng_gram_static.argtypes = [C.POINTER(vp), u32, u64, vp, u32, u64, vp, vp]
-            L.tng_static_scratch_limits.argtypes = [C.POINTER(u32), C.POINTER(u32)]
-            L.tng_static_scratch_limits.restype = None
         _lib = L
     return _lib
 
