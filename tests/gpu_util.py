@@ -6,6 +6,10 @@ import oracle
 from paper_1901_08227_b200 import tng, workloads
 
 
+def round_up4(d):
+    return (d + 3) // 4 * 4
+
+
 def to_np(t):
     return t.detach().cpu().numpy()
 
@@ -43,6 +47,8 @@ def make_oracle(d, M, K, codec, norm, **opts):
 def drifting_grads(seed, steps, M, d, device, ld=None, noise=0.3):
     """slowly drifting mean + per-worker noise, as (M, d) views with row stride ld"""
     traj = workloads.AR1Trajectory(seed, d, device=device, rho=0.95)
+    if ld is None:
+        ld = round_up4(d)
     for _ in range(steps):
         traj.advance()
         yield traj.worker_grads(M, noise, ld=ld)

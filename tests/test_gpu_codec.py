@@ -6,7 +6,7 @@ import pytest
 import torch
 
 import oracle
-from gpu_util import codes_np, make_ctx, same_values, to_np
+from gpu_util import codes_np, make_ctx, round_up4, same_values, to_np
 from paper_1901_08227_b200 import tng, workloads
 
 pytestmark = pytest.mark.gpu
@@ -17,7 +17,7 @@ NORMS = [tng.NORM_NONE, tng.NORM_DIFF, tng.NORM_QUOT]
 
 def run_both(d, M, codec, norm, B, scale_kind=0, s=7, seed=(3, 9), step=5, ld=None, kind="normal", ref_kind="near"):
     dev = "cuda"
-    g = workloads.random_grads(d * 7 + M, M, d, device=dev, ld=ld, kind=kind)
+    g = workloads.random_grads(d * 7 + M, M, d, device=dev, ld=ld or round_up4(d), kind=kind)
     if ref_kind == "near":
         ref = (g.mean(0) * 0.9 + 0.05 * workloads.normal((d,), 11, 1, dev)).contiguous()
     elif ref_kind == "zeros":
