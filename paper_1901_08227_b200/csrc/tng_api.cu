@@ -47,6 +47,7 @@ struct tng_ctx {
     const float* ref_cur = nullptr;   // reference of the last fusion (ref buffer or a ring slot)
     int last_mode = TNG_FUSE_LAST;
     bool last_had_stats = false;
+    bool last_solved = false;         // the last fusion ran the solve kernel (alpha lives on the device)
     // bookkeeping
     int device = 0, sm_count = 148;
     cudaStream_t last_stream = nullptr;
@@ -193,6 +194,7 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
     const int mode = c->effective_mode();
     c->last_mode = mode;
     c->last_had_stats = false;
+    c->last_solved = false;
     int launches = 0;
     if (c->k == 0) {   // empty trajectory: reference = zeros (initial state of Algorithm 1)
         TNG_CUDA(c, cudaMemsetAsync(c->ref_buf(), 0, c->d_pad * sizeof(float), st));
@@ -215,6 +217,7 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
     }
     if (tm) tm->mark(0, need_dots);
     TNG_CUDA(c, launch_solve(c->fb(), (int)c->k, mode, c->ridge, c->M, st, &launches));
+    c->last_solved = true;
     if (tm) tm->mark(1, true);
     TNG_CUDA(c, launch_combine(rows, (int)c->k, c->d, c->fb(), c->ref_buf(), c->sm_count, st, &launches));
     if (tm) tm->mark(2, true);
@@ -452,8 +455,8 @@ tng_status tng_stats(tng_ctx* c, tng_stats_t* out) {
     FuseBlock h;
     TNG_CUDA(c, cudaMemcpy(&h, c->fb(), sizeof h, cudaMemcpyDeviceToHost));
     const int mode = c->last_mode;
-    if (mode == TNG_FUSE_LAST || c->rounds == 0) {
-        out->alpha[0] = (c->k > 0 || c->rounds > 0) ? 1.0 : 0.0;
+    if (!c->last_solved) {
+        out->alpha[0] = (mode == TNG_FUSE_LAST && c->ref_cur && c->ref_cur != c->ref_buf()) ? 1.0 : 0.0;
     } else {
         for (int j = 0; j < TNG_MAX_HISTORY; ++j) out->alpha[j] = h.alpha64[j];
         out->solver_fallback = h.fallback;
