@@ -1,0 +1,350 @@
+#!/usr/bin/env python
+"""Benchmark of the TNG round (tng_step) on synthetic data shaped like a DNN-sized
+gradient stream: d = 2^27 fp32 coordinates, M = 8 workers, ring depth K = 8,
+quotient normalisation, ternary codes with one scale per 128 coordinates.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line.  `value` is GB/s of fp32 gradient (all M workers) pushed
+through whole rounds with inputs resident in device memory; `e2e` is the same
+metric through tng_step_host (pinned host buffers, copies inside the timed
+region); `roofline` describes the dominant kernel; `cpu_baseline` is the CPU
+oracle timed on a bounded sample of the same workload.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+from pathlib import Path
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+METRIC = "TNG step GB/s of fp32 gradient (all M workers)"
+UNIT = "GB/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+
+WORKLOADS = {
+    # name: d, M, K, norm, codec, block
+    "c5_dnn_stream": dict(d=1 << 27, M=8, K=8, norm="quot", codec="tern2", block=128, fuse="lsq"),
+    "c5_small": dict(d=1 << 22, M=8, K=8, norm="quot", codec="tern2", block=128, fuse="lsq"),
+}
+
+
+def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True):
+    """Bytes per coordinate each kernel of one round has to move (reads + writes)."""
+    wire = M * bits / 8.0 + 4.0 * M / block
+    per = {}
+    if fuse == "lsq":
+        per["dots"] = 4.0 * K + 4.0 * M
+        per["combine"] = 4.0 * K + 4.0
+    per["encode"] = 4.0 * M + 4.0 + wire
+    per["decode"] = wire + 4.0 + 4.0 + (4.0 if user_out else 0.0)
+    return per
+
+
+def measured_hbm_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured (MEASURED_PEAKS.json)"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons through NVML while the timed region runs."""
+
+    def __init__(self, index, period=0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period
+        self.samples, self.reasons = [], set()
+        self.max_mhz = None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            self.nv = pynvml
+            pynvml.nvmlInit()
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            "hw_slowdown": getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8),
+            "hw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40),
+            "sw_thermal_slowdown": getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20),
+            "sw_power_cap": getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4),
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for name, bit in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            time.sleep(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        self.join(timeout=2)
+        return {"sm_mhz": statistics.median(self.samples) if self.samples else None,
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+def enum_of(tng, cfg):
+    norm = {"none": tng.NORM_NONE, "diff": tng.NORM_DIFF, "quot": tng.NORM_QUOT}[cfg["norm"]]
+    codec = {"sign1": tng.CODEC_SIGN1, "tern2": tng.CODEC_TERN2, "qsgd4": tng.CODEC_QSGD4}[cfg["codec"]]
+    fuse = {"lsq": tng.FUSE_LSQ, "last": tng.FUSE_LAST, "mean": tng.FUSE_MEAN, "hindsight": tng.FUSE_HINDSIGHT}[cfg["fuse"]]
+    return norm, codec, fuse
+
+
+def config_dict(name, cfg, world):
+    return {"workload": name, "d": cfg["d"], "M": cfg["M"], "K": cfg["K"], "normalisation": cfg["norm"],
+            "codec": cfg["codec"], "block": cfg["block"], "fusion": cfg["fuse"],
+            "stream": "Student-t(nu=3) around an AR(1) mean (rho 0.99), 64 segments with LogUniform(1e-4,1e-1) scales",
+            "l2": "inputs exceed L2: every round streams the whole ring and all M gradient rows from HBM",
+            "sharding": "one process per GPU, each rank its own d coordinates" if world > 1 else "single GPU"}
+
+
+# --------------------------------------------------------------------------------------
+def run_reference(args, name, cfg):
+    """The CPU oracle, as it stands, timed on a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    import numpy as np
+
+    import oracle
+    from paper_1901_08227_b200 import tng, workloads
+    norm, codec, fuse = enum_of(tng, cfg)
+    M, K = cfg["M"], cfg["K"]
+    d_s = min(cfg["d"], 1 << 22)                  # the sample: the first 2^22 coordinates of the stream
+    stream = workloads.GradientStream(0, d_s, M, device="cpu")
+    orc = oracle.State(d_s, M, K, codec, norm, block=cfg["block"], fuse_mode=fuse)
+    for _ in range(K):
+        orc.push_reference(stream.advance().numpy())
+    batches = []
+    for _ in range(2):
+        stream.advance()
+        batches.append(stream.worker_grads().numpy())
+    for w in range(args.warmup):
+        orc.step(batches[w % 2])
+    t0 = time.perf_counter()
+    for s in range(args.steps):
+        orc.step(batches[s % 2])
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    value = M * d_s * 4 / dt / 1e9
+    cores = oracle.omp_threads()
+    sample = f"first {d_s} of {cfg['d']} coordinates per step (same stream recipe, M={M}, K={K})"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f32", "data": "synthetic", "config": config_dict(name, cfg, 1),
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+
+
+def time_cpu_baseline(cfg, enums, budget_s=12.0):
+    import oracle
+    from paper_1901_08227_b200 import workloads
+    norm, codec, fuse = enums
+    M, K = cfg["M"], cfg["K"]
+    d_s = min(cfg["d"], 1 << 22)
+    stream = workloads.GradientStream(0, d_s, M, device="cpu")
+    orc = oracle.State(d_s, M, K, codec, norm, block=cfg["block"], fuse_mode=fuse)
+    for _ in range(K):
+        orc.push_reference(stream.advance().numpy())
+    stream.advance()
+    g = stream.worker_grads().numpy()
+    orc.step(g)                                    # warm-up (page faults, thread pool)
+    n, t0 = 0, time.perf_counter()
+    while True:
+        orc.step(g)
+        n += 1
+        dt = time.perf_counter() - t0
+        if dt > budget_s or n >= 50:
+            break
+    per = dt / n
+    return {"value": M * d_s * 4 / per / 1e9, "unit": UNIT, "cores": oracle.omp_threads(), "kind": "oracle",
+            "sample": f"first {d_s} of {cfg['d']} coordinates per step, {n} steps, {per * 1e3:.1f} ms each"}
+
+
+# --------------------------------------------------------------------------------------
+def run_ours(args, name, cfg):
+    import torch
+    import torch.distributed as dist
+
+    from paper_1901_08227_b200 import tng, workloads
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local)
+    dev = torch.device("cuda", local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    tng.lib()                                       # fail loudly if libtng.so is missing
+
+    norm, codec, fuse = enum_of(tng, cfg)
+    d, M, K = cfg["d"], cfg["M"], cfg["K"]
+    bits = codec
+
+    cpu_baseline = None
+    if rank == 0 and not args.no_cpu_baseline:
+        cpu_baseline = time_cpu_baseline(cfg, (norm, codec, fuse))
+
+    # ---- inputs, resident in HBM: ring pre-filled with K past means, two gradient batches
+    stream = workloads.GradientStream(rank, d, M, device=dev)
+    ctx = tng.Context(d, M, K, codec, norm, block=cfg["block"], fuse_mode=fuse, timing=1, seed_lo=rank)
+    for _ in range(K):
+        ctx.push_reference(stream.advance())
+    batches = []
+    for _ in range(2):
+        stream.advance()
+        batches.append(stream.worker_grads())
+    out = torch.empty(d, device=dev)
+    del stream
+    torch.cuda.empty_cache()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for w in range(args.warmup):
+        ctx.step(batches[w % 2], out)
+    barrier()
+    st0 = ctx.stats()
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    ev0.record()
+    for s in range(args.steps):
+        ctx.step(batches[s % 2], out)
+    ev1.record()
+    barrier()
+    clocks = sampler.stop()
+    ms_total = ev0.elapsed_time(ev1)
+    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step = t.item() / args.steps
+    st1 = ctx.stats()
+    launches = st1.kernel_launches - st0.kernel_launches
+
+    # ---- per-kernel durations over the timed rounds (CUDA events recorded by the library on the same stream)
+    n0, n1 = st0.timed_rounds, st1.timed_rounds
+    def stage_ms(field):
+        return (getattr(st1, field) * n1 - getattr(st0, field) * n0) / max(n1 - n0, 1)
+    per_coord = algorithmic_bytes_per_coord(M, K, bits, cfg["block"], cfg["fuse"])
+    peak, peak_src = measured_hbm_peak()
+    kernels = {}
+    for kname, field in (("dots", "ms_dots"), ("combine", "ms_combine"), ("encode", "ms_encode"), ("decode", "ms_decode")):
+        if kname not in per_coord:
+            continue
+        ms = stage_ms(field)
+        gbs = per_coord[kname] * d / (ms * 1e-3) / 1e9 if ms > 0 else None
+        kernels[kname] = {"ms": ms, "bytes_per_coord": per_coord[kname], "GBps": gbs, "frac_of_measured": gbs / peak if gbs else None}
+    kernels["solve"] = {"ms": stage_ms("ms_solve")}
+    dominant = max((k for k in kernels if "bytes_per_coord" in kernels[k]), key=lambda k: kernels[k]["ms"])
+    traffic = {"dots": None, "combine": None, "encode": None, "decode": None}.get(dominant)
+    roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["GBps"], "peak": peak, "unit": "GB/s",
+                "frac": kernels[dominant]["frac_of_measured"], "peak_source": peak_src, "traffic": traffic,
+                "algorithmic_bytes_per_launch": per_coord[dominant] * d}
+    step_bytes = sum(per_coord.values()) * d
+    step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
+
+    # ---- end to end: host buffers through tng_step_host, copies inside the timed region
+    e2e = None
+    if not args.no_e2e:
+        ctx_h = tng.Context(d, M, K, codec, norm, block=cfg["block"], fuse_mode=fuse, host_staging=1, seed_lo=rank)
+        for j in range(K):
+            ctx_h.push_reference(ctx.history(K - 1 - j))
+        g_host = torch.empty((M, d), dtype=torch.float32).pin_memory()
+        g_host.copy_(batches[0])
+        o_host = torch.empty(d, dtype=torch.float32).pin_memory()
+        e2e_steps = max(1, min(args.steps, args.e2e_steps))
+        for _ in range(2):
+            ctx_h.step_host(g_host, o_host)
+        barrier()
+        t0 = time.perf_counter()
+        for _ in range(e2e_steps):
+            ctx_h.step_host(g_host, o_host)
+        torch.cuda.synchronize()
+        dt = torch.tensor([(time.perf_counter() - t0) / e2e_steps], dtype=torch.float64, device=dev)
+        if world > 1:
+            dist.all_reduce(dt, op=dist.ReduceOp.MAX)
+        e2e = {"value": world * M * d * 4 / dt.item() / 1e9, "unit": UNIT, "h2d_bytes_per_step": M * d * 4,
+               "d2h_bytes_per_step": d * 4, "steps": e2e_steps, "ms_per_step": dt.item() * 1e3,
+               "api": "tng_step_host (pinned host rows -> device staging -> round -> aggregate back to host)"}
+        ctx_h.close()
+        del g_host, o_host
+
+    if rank == 0:
+        value = world * M * d * 4 / (ms_step * 1e-3) / 1e9
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic", "config": config_dict(name, cfg, world), "clocks": clocks, "e2e": e2e,
+            "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu_baseline,
+            "coords_per_s": world * M * d / (ms_step * 1e-3),
+            "bits_per_coord": st1.bits_per_coord,
+            "step_hbm": {"algorithmic_bytes_per_coord": sum(per_coord.values()), "GBps": step_gbs,
+                         "frac_of_measured": step_gbs / peak, "frac_of_nominal_8TBps": step_gbs / NOMINAL_HBM_GBS},
+            "kernels": kernels, "cnz": st1.cnz, "solver_fallback": int(st1.solver_fallback),
+            "nonfinite_scales": int(st1.nonfinite_scales),
+        }
+        print(json.dumps(line), flush=True)
+    ctx.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="c5_dnn_stream", choices=sorted(WORKLOADS))
+    ap.add_argument("--e2e-steps", type=int, default=5)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    cfg = WORKLOADS[args.workload]
+    if args.impl == "reference":
+        args.steps = 3 if args.steps is None else args.steps
+        args.warmup = 1 if args.warmup is None else args.warmup
+        run_reference(args, args.workload, cfg)
+        return
+    args.steps = 200 if args.steps is None else args.steps
+    args.warmup = 5 if args.warmup is None else max(args.warmup, 0)
+    run_ours(args, args.workload, cfg)
+
+
+if __name__ == "__main__":
+    main()
