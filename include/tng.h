@@ -149,6 +149,32 @@ tng_status tng_reference(tng_ctx* ctx, const float** ref_dev);
 /* h_{j+1}: j = 0 is the newest stored aggregate; j < k. */
 tng_status tng_history(tng_ctx* ctx, uint32_t j, const float** vec_dev);
 
+/* ---- fusion statistics without any allocation ------------------------------- */
+/* (No counterpart in the paper: this is a packaging of the statistics pass of tng_fuse.)
+ * For callers that cannot allocate device memory -- a process whose device memory is
+ * owned by its own pool, a steady-state loop that must stay away from cudaMalloc (it
+ * synchronises the device and may fail), a plug-in that only receives pointers -- this
+ * computes, for k history vectors and M gradient rows,
+ *   out[0 .. k*k)      G[a][b] = <h_a, h_b>            (row-major, both triangles)
+ *   out[k*k .. k*k+k)  c[a]    = <h_a, mean_m g^m>
+ *   out[k*k+k]         (1/M) sum_m ||g^m||^2
+ * (doubles) with the same kernel tng_fuse uses.  The per-CTA partial sums and the arrival
+ * counter that kernel needs live in a fixed array inside the library image
+ * (TNG_STATIC_SCRATCH_BYTES per GPU that loads the library, held until the process
+ * exits), so the call performs no cudaMalloc/cudaFree and uses no allocating routine.
+ * rows_dev is a HOST array of k device pointers (16-byte aligned vectors of d floats);
+ * grads_dev/ld as in tng_step; out_dev: k*k+k+1 doubles, caller-owned device memory.
+ * Limits: 1 <= k <= TNG_STATIC_MAX_HISTORY, M <= TNG_MAX_WORKERS; beyond them the call
+ * returns TNG_ERR_UNSUPPORTED and launches nothing.
+ * The first call on each device looks up the array's device address (with that device
+ * current); make that first call outside any stream capture.  All calls share the one
+ * array: it is cleared where it must start at zero, but two calls that overlap on the
+ * GPU (different streams, different threads) race and give wrong sums. */
+#define TNG_STATIC_MAX_HISTORY 8
+#define TNG_STATIC_SCRATCH_BYTES (320 * 1024)
+tng_status tng_gram_static(const float* const* rows_dev, uint32_t k, uint64_t d, const float* grads_dev,
+                           uint32_t M, uint64_t ld, double* out_dev, void* stream);
+
 /* Synchronises the context's last stream and fills *out. */
 tng_status tng_stats(tng_ctx* ctx, tng_stats_t* out);
 const char* tng_status_string(tng_status s);

@@ -10,7 +10,7 @@ PKG = Path(__file__).resolve().parent
 ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libtng.so"
-SOURCES = ["tng_api.cu", "tng_fuse.cu", "tng_codec.cu", "tng_producers.cu"]
+SOURCES = ["tng_api.cu", "tng_fuse.cu", "tng_codec.cu", "tng_producers.cu", "tng_static.cu"]
 HEADERS = [CSRC / "tng_device.cuh", CSRC / "tng_internal.h", ROOT / "include" / "tng.h"]
 
 NVCC_FLAGS = [

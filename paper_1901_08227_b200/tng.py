@@ -26,7 +26,7 @@ EXPORTS = [
     "tng_push_reference", "tng_step", "tng_step_host", "tng_fuse", "tng_encode", "tng_decode_aggregate",
     "tng_wire", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
     "tng_logistic_scratch_floats", "tng_logistic_grad", "tng_logistic_loss", "tng_rosenbrock_grad",
-    "tng_rosenbrock_value", "tng_sgd_update",
+    "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static",
 ]
 
 
@@ -86,6 +86,7 @@ def lib():
         L.tng_rosenbrock_grad.argtypes = [vp, u64, vp, u32, u64, vp, vp]
         L.tng_rosenbrock_value.argtypes = [vp, u64, vp, vp]
         L.tng_sgd_update.argtypes = [vp, vp, u64, f32, vp]
+        L.tng_gram_static.argtypes = [C.POINTER(vp), u32, u64, vp, u32, u64, vp, vp]
         _lib = L
     return _lib
 
@@ -241,6 +242,18 @@ class _DeviceView:
 def _view(ptr, shape, dtype):
     typestr = {torch.float32: "<f4", torch.int32: "<i4"}[dtype]
     return torch.as_tensor(_DeviceView(ptr, shape, typestr), device="cuda")
+
+
+def gram_static(rows, grads, out):
+    """tng_gram_static: Gram / rhs / mean squared norm of `rows` (list of (d,) CUDA tensors,
+    newest first) against the (M, d) gradient rows, into `out` (k*k+k+1 float64 on the GPU).
+    Allocates nothing on the device."""
+    k = len(rows)
+    arr = (C.c_void_p * max(k, 1))(*[_dev(r) for r in rows])
+    p, ld = _rows(grads)
+    d = rows[0].numel() if k else 0
+    _check(lib().tng_gram_static(arr, k, d, p, grads.shape[0], ld, _dev(out, torch.float64), _stream()), "tng_gram_static")
+    return out
 
 
 # ---- producers -------------------------------------------------------------------------
