@@ -34,6 +34,7 @@ FALLBACK_HBM_GBS = 6650.0
 WORKLOADS = {
     # name: d, M, K, norm, codec, block
     "c5_dnn_stream": dict(d=1 << 27, M=8, K=8, norm="quot", codec="tern2", block=128, fuse="lsq"),
+    "c5_mid": dict(d=1 << 24, M=8, K=8, norm="quot", codec="tern2", block=128, fuse="lsq"),   # profiler-sized
     "c5_small": dict(d=1 << 22, M=8, K=8, norm="quot", codec="tern2", block=128, fuse="lsq"),
 }
 
