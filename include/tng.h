@@ -73,6 +73,7 @@ typedef enum {
 
 #define TNG_MAX_WORKERS 64
 #define TNG_MAX_HISTORY 16
+#define TNG_MAX_COORDS (1ull << 31) /* d; a row stride must stay below 2^32 floats */
 #define TNG_TILE 128 /* coordinates per wire tile */
 
 /* Plain-old-data snapshot filled by tng_stats. */
@@ -89,7 +90,7 @@ typedef struct {
     double grad_sq;          /* (1/M) sum_m ||g^m||^2 of the last fusion */
     double cnz;              /* estimate of C_nz = sum_m||g^m - r||^2 / sum_m||g^m||^2; NaN if unknown */
     uint32_t solver_fallback;   /* 1 = last solve hit a bad pivot and used alpha = e_1 */
-    uint32_t reserved;
+    uint32_t pipeline_error;    /* nonzero: a bounded wait inside a staged kernel gave up (results invalid) */
     uint64_t nonfinite_scales;  /* block scales that were NaN/Inf since creation */
     uint64_t kernel_launches;   /* kernels launched by this context since creation */
     /* mean milliseconds per round of each stage over the rounds timed so far
@@ -99,7 +100,7 @@ typedef struct {
 } tng_stats_t;
 
 /* ---- lifetime --------------------------------------------------------------- */
-/* d >= 1 coordinates, 1 <= M <= 64 workers, ring depth 1 <= K <= 16.  Host only. */
+/* 1 <= d <= TNG_MAX_COORDS coordinates, 1 <= M <= 64 workers, ring depth 1 <= K <= 16.  Host only. */
 tng_status tng_create(tng_ctx** out, uint64_t d, uint32_t M, uint32_t K, tng_codec codec,
                       tng_norm_mode norm);
 /* Waits for the context's last stream, frees what the library allocated.  NULL is allowed. */
@@ -175,7 +176,8 @@ tng_status tng_history(tng_ctx* ctx, uint32_t j, const float** vec_dev);
 tng_status tng_gram_static(const float* const* rows_dev, uint32_t k, uint64_t d, const float* grads_dev,
                            uint32_t M, uint64_t ld, double* out_dev, void* stream);
 
-/* Synchronises the context's last stream and fills *out. */
+/* Synchronises the context's last stream and fills *out.  Returns TNG_ERR_CUDA if a staged
+ * kernel reported a pipeline error, TNG_ERR_NONFINITE if new non-finite scales were counted. */
 tng_status tng_stats(tng_ctx* ctx, tng_stats_t* out);
 const char* tng_status_string(tng_status s);
 /* cudaError_t value of the last failing CUDA call seen by this context (0 if none). */

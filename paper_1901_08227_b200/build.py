@@ -11,7 +11,7 @@ ROOT = PKG.parent
 CSRC = PKG / "csrc"
 LIB = PKG / "libtng.so"
 SOURCES = ["tng_api.cu", "tng_fuse.cu", "tng_codec.cu", "tng_producers.cu", "tng_static.cu"]
-HEADERS = [CSRC / "tng_device.cuh", CSRC / "tng_internal.h", ROOT / "include" / "tng.h"]
+HEADERS = [CSRC / "tng_device.cuh", CSRC / "tng_pipeline.cuh", CSRC / "tng_internal.h", ROOT / "include" / "tng.h"]
 
 NVCC_FLAGS = [
     "-O3", "-std=c++17", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",

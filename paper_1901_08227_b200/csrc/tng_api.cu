@@ -146,7 +146,7 @@ tng_status ensure_ready(tng_ctx* c, cudaStream_t st) {
 }
 
 tng_status check_rows(const tng_ctx* c, const float* p, uint64_t ld) {
-    if (!p || !aligned16(p) || ld < c->d || (ld % 4) != 0) return TNG_ERR_INVALID_ARG;
+    if (!p || !aligned16(p) || ld < c->d || (ld % 4) != 0 || ld > 0xFFFFFFFCull) return TNG_ERR_INVALID_ARG;
     return TNG_OK;
 }
 
@@ -190,7 +190,10 @@ struct StageTimer {
 };
 
 // ---- the stages -----------------------------------------------------------------------
-tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st, StageTimer* tm) {
+// `defer` (may be nullptr): when the encode pass can build the reference itself, the combine
+// launch is skipped and *defer describes the combination for launch_encode.
+tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st, StageTimer* tm, RefFusion* defer) {
+    if (defer) defer->k = 0;
     const int mode = c->effective_mode();
     c->last_mode = mode;
     c->last_had_stats = false;
@@ -219,16 +222,25 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
     TNG_CUDA(c, launch_solve(c->fb(), (int)c->k, mode, c->ridge, c->M, st, &launches));
     c->last_solved = true;
     if (tm) tm->mark(1, true);
-    TNG_CUDA(c, launch_combine(rows, (int)c->k, c->d, c->fb(), c->ref_buf(), c->sm_count, st, &launches));
-    if (tm) tm->mark(2, true);
+    if (defer && encode_can_fuse_reference(c->geom)) {
+        for (uint32_t j = 0; j < c->k; ++j) defer->rows[j] = rows[j];
+        defer->k = (int)c->k;
+        defer->alpha = c->fb()->alpha32;
+        defer->ref_out = c->ref_buf();
+        if (tm) tm->mark(2, false);
+    } else {
+        TNG_CUDA(c, launch_combine(rows, (int)c->k, c->d, c->fb(), c->ref_buf(), c->sm_count, st, &launches));
+        if (tm) tm->mark(2, true);
+    }
     c->ref_cur = c->ref_buf();
     c->launches += (uint64_t)launches;
     return TNG_OK;
 }
 
-tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* ref, uint32_t step, cudaStream_t st) {
+tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* ref, const RefFusion* fusion, uint32_t step,
+                     cudaStream_t st) {
     int launches = 0;
-    TNG_CUDA(c, launch_encode(c->geom, grads, ld, ref, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
+    TNG_CUDA(c, launch_encode(c->geom, grads, ld, ref, fusion, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
                               c->fb(), c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
@@ -243,9 +255,10 @@ tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, c
 
 tng_status step_impl(tng_ctx* c, const float* grads, uint64_t ld, float* out, cudaStream_t st) {
     StageTimer tm(c, st);
-    tng_status s = do_fuse(c, grads, ld, st, &tm);
+    RefFusion fusion;
+    tng_status s = do_fuse(c, grads, ld, st, &tm, &fusion);
     if (s != TNG_OK) return s;
-    s = do_encode(c, grads, ld, c->ref_cur, (uint32_t)c->rounds, st);
+    s = do_encode(c, grads, ld, c->ref_cur, &fusion, (uint32_t)c->rounds, st);
     if (s != TNG_OK) return s;
     tm.mark(3, true);
     // the decoded aggregate goes straight into the next ring slot (and to the caller's buffer)
@@ -267,7 +280,7 @@ extern "C" {
 tng_status tng_create(tng_ctx** out, uint64_t d, uint32_t M, uint32_t K, tng_codec codec, tng_norm_mode norm) {
     if (!out) return TNG_ERR_INVALID_ARG;
     *out = nullptr;
-    if (d < 1 || d > (1ull << 40) || M < 1 || M > TNG_MAX_WORKERS || K < 1 || K > TNG_MAX_HISTORY) return TNG_ERR_INVALID_ARG;
+    if (d < 1 || d > TNG_MAX_COORDS || M < 1 || M > TNG_MAX_WORKERS || K < 1 || K > TNG_MAX_HISTORY) return TNG_ERR_INVALID_ARG;
     if (codec != TNG_CODEC_SIGN1 && codec != TNG_CODEC_TERN2 && codec != TNG_CODEC_QSGD4) return TNG_ERR_INVALID_ARG;
     if (norm != TNG_NORM_NONE && norm != TNG_NORM_DIFF && norm != TNG_NORM_QUOT) return TNG_ERR_INVALID_ARG;
     tng_ctx* c = new (std::nothrow) tng_ctx();
@@ -366,7 +379,7 @@ tng_status tng_step(tng_ctx* c, const float* grads_dev, uint64_t ld, float* agg_
 }
 
 tng_status tng_step_host(tng_ctx* c, const float* grads_host, uint64_t ld, float* agg_out_host, void* stream) {
-    if (!c || !grads_host || !agg_out_host || ld < c->d) return TNG_ERR_INVALID_ARG;
+    if (!c || !grads_host || !agg_out_host || ld < c->d || ld > 0xFFFFFFFCull) return TNG_ERR_INVALID_ARG;
     if (!c->host_staging) return TNG_ERR_STATE;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     tng_status s = ensure_ready(c, st);
@@ -387,7 +400,7 @@ tng_status tng_fuse(tng_ctx* c, const float* grads_dev, uint64_t ld, void* strea
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
-    return do_fuse(c, grads_dev, ld, st, nullptr);
+    return do_fuse(c, grads_dev, ld, st, nullptr, nullptr);
 }
 
 tng_status tng_encode(tng_ctx* c, const float* grads_dev, uint64_t ld, const float* ref_dev, uint32_t step, void* stream) {
@@ -400,7 +413,7 @@ tng_status tng_encode(tng_ctx* c, const float* grads_dev, uint64_t ld, const flo
     if (s != TNG_OK) return s;
     const float* ref = ref_dev ? ref_dev : c->ref_cur;
     if (!ref && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;   // no fusion has produced a reference yet
-    return do_encode(c, grads_dev, ld, ref, step, st);
+    return do_encode(c, grads_dev, ld, ref, nullptr, step, st);
 }
 
 tng_status tng_decode_aggregate(tng_ctx* c, const float* ref_dev, float* out_dev, void* stream) {
@@ -470,12 +483,14 @@ tng_status tng_stats(tng_ctx* c, tng_stats_t* out) {
         }
     }
     out->nonfinite_scales = h.nonfinite;
+    out->pipeline_error = h.pipe_error;
     out->timed_rounds = c->timed_rounds;
     if (c->timed_rounds) {
         const double n = (double)c->timed_rounds;
         out->ms_dots = c->ms_sum[0] / n; out->ms_solve = c->ms_sum[1] / n; out->ms_combine = c->ms_sum[2] / n;
         out->ms_encode = c->ms_sum[3] / n; out->ms_decode = c->ms_sum[4] / n;
     }
+    if (h.pipe_error != 0) return TNG_ERR_CUDA;
     if (h.nonfinite > c->nonfinite_reported) {
         c->nonfinite_reported = h.nonfinite;
         return TNG_ERR_NONFINITE;

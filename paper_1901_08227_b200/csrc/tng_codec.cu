@@ -11,13 +11,18 @@
 // decode follows Algorithm 1's averaging step with the reference put back.
 #include "tng_device.cuh"
 #include "tng_internal.h"
+#include "tng_pipeline.cuh"
 
 namespace tng {
 
 namespace {
 
 enum { kPhaseFused = 0, kPhaseStat = 1, kPhaseQuant = 2 };
+constexpr int kCodecThreads = 256;
+constexpr int kWorkerBatch = 4;   // gradient rows whose loads are in flight together
 
+// Row strides are 32-bit element counts (the entry points reject longer rows), so that
+// "base + m * stride" is one 32 x 32 -> 64-bit multiply-add per address.
 struct EncodeArgs {
     const float* grads;
     const float* ref;
@@ -25,117 +30,316 @@ struct EncodeArgs {
     float* scales;
     float* tile_stat;
     unsigned long long* nonfinite;
-    uint64_t ld, d, ntile, nblk, block, wpw;
-    uint32_t M, step, seed_lo, seed_hi;
+    uint32_t* pipe_error;
+    uint64_t d, ntile, block;
+    uint64_t tile_begin;   // first tile this launch handles (the staged kernel takes the ones before it)
+    uint32_t ld, nblk, wpw;
+    uint32_t M, step;
+    uint32_t pow24;    // 1 << 24 as a run-time value: x >> 8 is taken as umulhi(x, 2^24)
+    uint32_t rk[20];   // Philox round keys (key + r * Weyl), computed once on the host
     int levels;
     float quot_eps;
+    // reference fusion inside the encode pass: r = sum_j alpha[j] hist[j] is computed per tile
+    // (fp32 fma chain, j ascending) and written to ref_out, instead of being read from `ref`
+    const float* hist[kMaxK];
+    const float* alpha;
+    float* ref_out;
+    int hist_k;
 };
 
-template <int CODEC, int NORM, int SCALE, int PHASE>
-__device__ __forceinline__ void encode_worker(const EncodeArgs& a, const float4 g, const float4 op,
-                                              const uint32_t m, const uint64_t T, const uint64_t blk,
-                                              const int lane, const uint32_t valid) {
+// max(|a|, |b|) that returns NaN if either is NaN
+__device__ __forceinline__ float absmax_nan2(float a, float b) {
+    float r;
+    asm("max.NaN.f32 %0, %1, %2;" : "=f"(r) : "f"(fabsf(a)), "f"(fabsf(b)));
+    return r;
+}
+
+// One worker's share of one tile.  A scale that is zero, NaN or infinite needs no
+// special case in the quantisers: u*0 < 0, NaN < x and inf < x are all false, and
+// (int)NaN is 0, so every symbol of such a block comes out as the zero symbol.
+// Returns the bit pattern of the scale it used (for the non-finite bookkeeping).
+//
+// The integer/logic pipe is the busy one in this kernel (Philox xors, compares,
+// ballots), so work that can run on the multiplier pipe is put there: addresses are
+// 32 x 32 -> 64 multiply-adds and the uniform's shift is a high multiply.
+template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL>
+__device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const float4 g, const float4 op,
+                                                  const uint32_t m, const uint64_t T, const uint32_t q_lo,
+                                                  const uint32_t q_hi, const uint64_t blk, const int lane,
+                                                  const uint32_t valid) {
     // ---- normalise: v = g - r (Eq. 2), v = g * (1/den) (Eq. 3), or v = g
-    float v0, v1, v2, v3;
+    float v[4];
     if (NORM == TNG_NORM_DIFF) {
-        v0 = __fsub_rn(g.x, op.x); v1 = __fsub_rn(g.y, op.y); v2 = __fsub_rn(g.z, op.z); v3 = __fsub_rn(g.w, op.w);
+        v[0] = __fsub_rn(g.x, op.x); v[1] = __fsub_rn(g.y, op.y); v[2] = __fsub_rn(g.z, op.z); v[3] = __fsub_rn(g.w, op.w);
     } else if (NORM == TNG_NORM_QUOT) {
-        v0 = __fmul_rn(g.x, op.x); v1 = __fmul_rn(g.y, op.y); v2 = __fmul_rn(g.z, op.z); v3 = __fmul_rn(g.w, op.w);
+        v[0] = __fmul_rn(g.x, op.x); v[1] = __fmul_rn(g.y, op.y); v[2] = __fmul_rn(g.z, op.z); v[3] = __fmul_rn(g.w, op.w);
     } else {
-        v0 = g.x; v1 = g.y; v2 = g.z; v3 = g.w;
+        v[0] = g.x; v[1] = g.y; v[2] = g.z; v[3] = g.w;
     }
     // ---- scale of the block
     float R;
     if (PHASE != kPhaseQuant) {
-        const float stat = (SCALE == 0) ? warp_absmax(v0, v1, v2, v3) : warp_sumsq_tree(v0, v1, v2, v3);
+        float stat;
+        if (SCALE == 0) {
+            const float mx = absmax_nan2(absmax_nan2(v[0], v[1]), absmax_nan2(v[2], v[3]));
+            // non-negative floats and NaNs order like their bit patterns
+            stat = __uint_as_float(__reduce_max_sync(kFullMask, __float_as_uint(mx)));
+        } else {
+            stat = warp_sumsq_tree(v[0], v[1], v[2], v[3]);
+        }
         if (PHASE == kPhaseStat) {
             if (lane == 0) a.tile_stat[(uint64_t)m * a.ntile + T] = stat;
-            return;
+            return 0u;
         }
         R = (SCALE == 0) ? stat : __fsqrt_rn(stat);
-        if (lane == 0) {
-            a.scales[(uint64_t)m * a.nblk + T] = R;
-            if (!(R < __int_as_float(0x7f800000))) atomicAdd(a.nonfinite, 1ull);   // NaN or +inf
-        }
     } else {
         R = __ldg(a.scales + (uint64_t)m * a.nblk + blk);
     }
-    const bool ok = !scale_is_bad(R);
 
     // ---- stochastic rounding: one Philox call per lane, word c for coordinate 4j+c
-    const uint64_t q = T * 32u + (uint32_t)lane;
-    const uint4 x = philox4x32_10((uint32_t)q, (uint32_t)(q >> 32), m, a.step, a.seed_lo, a.seed_hi);
-    const float u[4] = {uniform24(x.x), uniform24(x.y), uniform24(x.z), uniform24(x.w)};
-    const float v[4] = {v0, v1, v2, v3};
-
-    uint32_t mine = 0;
+    const uint4 x = philox4x32_10_rk(q_lo, q_hi, m, a.step, a.rk);
+    const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+    constexpr int kWords = 4 * CODEC;
+    uint32_t w[kWords];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
-        const bool live = ok && ((valid >> c) & 1u);
+        // u = (x >> 8) * 2^-24
+        const float u = __fmul_rn(__uint2float_rn(__umulhi(xs[c], a.pow24)), 0x1p-24f);
+        const bool live = FULL || ((valid >> c) & 1u);
         if (CODEC == TNG_CODEC_TERN2) {
             // nonzero with probability |v|/R  <=>  u*R < |v|
-            const bool nz = live && (__fmul_rn(u[c], R) < fabsf(v[c]));
+            const bool nz = live && (__fmul_rn(u, R) < fabsf(v[c]));
             const bool neg = nz && (v[c] < 0.0f);
-            const uint32_t w0 = __ballot_sync(kFullMask, nz);
-            const uint32_t w1 = __ballot_sync(kFullMask, neg);
-            if (lane == c * 2 + 0) mine = w0;
-            if (lane == c * 2 + 1) mine = w1;
+            w[c * 2 + 0] = __ballot_sync(kFullMask, nz);
+            w[c * 2 + 1] = __ballot_sync(kFullMask, neg);
         } else if (CODEC == TNG_CODEC_SIGN1) {
             // +R with probability (1 + v/R)/2  <=>  u*R < v/2 + R/2
             const float thr = __fadd_rn(__fmul_rn(0.5f, v[c]), __fmul_rn(0.5f, R));
-            const bool plus = live && (__fmul_rn(u[c], R) < thr);
-            const uint32_t w0 = __ballot_sync(kFullMask, plus);
-            if (lane == c) mine = w0;
+            const bool plus = live && (__fmul_rn(u, R) < thr);
+            w[c] = __ballot_sync(kFullMask, plus);
         } else {
             // s-level: a = (|v|/R) s; level floor(a) (+1 with probability frac(a))
             const float qv = __fdiv_rn(fabsf(v[c]), R);
             const float av = __fmul_rn(qv, (float)a.levels);
             const float lv = floorf(av);
             const float fv = __fsub_rn(av, lv);
-            int L = live ? ((int)lv + ((u[c] < fv) ? 1 : 0)) : 0;
+            const int L = live ? ((int)lv + ((u < fv) ? 1 : 0)) : 0;
             const bool neg = (L > 0) && (v[c] < 0.0f);
-            const uint32_t w0 = __ballot_sync(kFullMask, L & 1);
-            const uint32_t w1 = __ballot_sync(kFullMask, L & 2);
-            const uint32_t w2 = __ballot_sync(kFullMask, L & 4);
-            const uint32_t w3 = __ballot_sync(kFullMask, neg);
-            if (lane == c * 4 + 0) mine = w0;
-            if (lane == c * 4 + 1) mine = w1;
-            if (lane == c * 4 + 2) mine = w2;
-            if (lane == c * 4 + 3) mine = w3;
+            w[c * 4 + 0] = __ballot_sync(kFullMask, L & 1);
+            w[c * 4 + 1] = __ballot_sync(kFullMask, L & 2);
+            w[c * 4 + 2] = __ballot_sync(kFullMask, L & 4);
+            w[c * 4 + 3] = __ballot_sync(kFullMask, neg);
         }
     }
-    if (lane < 4 * CODEC) __stcs(a.codes + (uint64_t)m * a.wpw + T * (4u * CODEC) + lane, mine);
+    // every lane holds all words of the tile; lane 0 writes them (and the scale)
+    if (lane == 0) {
+        uint4* dst = reinterpret_cast<uint4*>(a.codes + ((uint64_t)m * a.wpw + T * (uint64_t)kWords));
+#pragma unroll
+        for (int q4 = 0; q4 < CODEC; ++q4) __stcs(dst + q4, make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]));
+        if (PHASE == kPhaseFused) a.scales[(uint64_t)m * a.nblk + T] = R;
+    }
+    return __float_as_uint(R);
 }
 
-template <int CODEC, int NORM, int SCALE, int PHASE>
-__global__ void __launch_bounds__(256) encode_kernel(const EncodeArgs a) {
-    const int lane = threadIdx.x & 31;
-    const uint64_t warps_per_cta = blockDim.x >> 5;
-    const uint64_t nwarps = (uint64_t)gridDim.x * warps_per_cta;
-    for (uint64_t T = (uint64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5); T < a.ntile; T += nwarps) {
-        const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
-        uint32_t valid = 0;
+template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL, bool FUSEREF>
+__device__ __forceinline__ void encode_tile(const EncodeArgs& a, const float* s_alpha, const uint64_t T, const int lane) {
+    const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
+    uint32_t valid = 0xFu;
+    if (!FULL) {
+        valid = 0;
 #pragma unroll
         for (int c = 0; c < 4; ++c) valid |= (i0 + c < a.d) ? (1u << c) : 0u;
-        float4 op = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+    const float* gp = a.grads + i0;
+    auto load_row = [&](uint32_t m) -> float4 {
+        const float* row = gp + (uint64_t)m * a.ld;
+        return FULL ? __ldcs(reinterpret_cast<const float4*>(row)) : load4_stream(row - i0, i0, a.d);
+    };
+    // the first batch of gradient rows is requested before anything is computed
+    float4 g[kWorkerBatch];
+#pragma unroll
+    for (int k = 0; k < kWorkerBatch; ++k)
+        if ((uint32_t)k < a.M) g[k] = load_row(k);
+
+    float4 op = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (NORM != TNG_NORM_NONE) {
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (FUSEREF) {
+            for (int j0 = 0; j0 < a.hist_k; j0 += 4) {
+                float4 h[4];
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj)
+                    if (j0 + jj < a.hist_k)
+                        h[jj] = FULL ? __ldcs(reinterpret_cast<const float4*>(a.hist[j0 + jj] + i0)) : load4_stream(a.hist[j0 + jj], i0, a.d);
+#pragma unroll
+                for (int jj = 0; jj < 4; ++jj)
+                    if (j0 + jj < a.hist_k) {
+                        const float al = s_alpha[j0 + jj];
+                        r.x = __fmaf_rn(al, h[jj].x, r.x); r.y = __fmaf_rn(al, h[jj].y, r.y);
+                        r.z = __fmaf_rn(al, h[jj].z, r.z); r.w = __fmaf_rn(al, h[jj].w, r.w);
+                    }
+            }
+            if (FULL) *reinterpret_cast<float4*>(a.ref_out + i0) = r;
+            else store4(a.ref_out, i0, a.d, r);
+        } else if (a.ref) {
+            r = FULL ? *reinterpret_cast<const float4*>(a.ref + i0) : load4(a.ref, i0, a.d);
+        }
         if (NORM == TNG_NORM_DIFF) {
-            if (a.ref) op = load4(a.ref, i0, a.d);
-        } else if (NORM == TNG_NORM_QUOT) {
-            float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (a.ref) r = load4(a.ref, i0, a.d);
+            op = r;
+        } else {
             const float4 den = quot_den4(r, a.quot_eps);
             op = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z),
                              __fdiv_rn(1.0f, den.w));
         }
-        const uint64_t blk = (PHASE == kPhaseQuant) ? (T * kTile) / a.block : T;
-        for (uint32_t m0 = 0; m0 < a.M; m0 += 4) {
-            float4 g[4];
+    }
+    const uint64_t blk = (PHASE == kPhaseQuant) ? (T * kTile) / a.block : T;
+    const uint64_t q = T * 32u + (uint32_t)lane;                 // Philox counter of the lane's four coordinates
+    const uint32_t q_lo = (uint32_t)q, q_hi = (uint32_t)(q >> 32);
+    uint32_t rmax = 0;                                           // largest scale bit pattern of the tile
+    // batches of rows; the next batch is in flight while the current one is encoded
+    const uint32_t m_batched = a.M - a.M % kWorkerBatch;
+    for (uint32_t m0 = 0; m0 < m_batched; m0 += kWorkerBatch) {
+        float4 gn[kWorkerBatch];
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (m0 + k < a.M) g[k] = load4_stream(a.grads + (uint64_t)(m0 + k) * a.ld, i0, a.d);
+        for (int k = 0; k < kWorkerBatch; ++k)
+            if (m0 + kWorkerBatch + k < a.M) gn[k] = load_row(m0 + kWorkerBatch + k);
 #pragma unroll
-            for (int k = 0; k < 4; ++k)
-                if (m0 + k < a.M) encode_worker<CODEC, NORM, SCALE, PHASE>(a, g[k], op, m0 + k, T, blk, lane, valid);
+        for (int k = 0; k < kWorkerBatch; ++k)
+            rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, PHASE, FULL>(a, g[k], op, m0 + k, T, q_lo, q_hi, blk, lane, valid));
+#pragma unroll
+        for (int k = 0; k < kWorkerBatch; ++k) g[k] = gn[k];
+    }
+#pragma unroll
+    for (int k = 0; k < kWorkerBatch - 1; ++k)
+        if (m_batched + k < a.M)
+            rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, PHASE, FULL>(a, g[k], op, m_batched + k, T, q_lo, q_hi, blk, lane, valid));
+    // NaN or +inf scales are rare: only then count them, from the scales just written
+    if (PHASE == kPhaseFused && rmax >= 0x7f800000u && lane == 0) {
+        unsigned long long bad = 0;
+        for (uint32_t m = 0; m < a.M; ++m) bad += (__float_as_uint(a.scales[(uint64_t)m * a.nblk + T]) >= 0x7f800000u) ? 1ull : 0ull;
+        atomicAdd(a.nonfinite, bad);
+    }
+}
+
+// Persistent grid: warp w of the grid takes tiles w, w + nwarps, ...; at any moment the
+// grid works on one contiguous window of every input row.  Only the last tile can be
+// ragged; it runs the bounds-checked instantiation.
+template <int CODEC, int NORM, int SCALE, int PHASE, bool FUSEREF>
+__global__ void __launch_bounds__(kCodecThreads, 2) encode_kernel(const EncodeArgs a) {
+    __shared__ float s_alpha[kMaxK];
+    if (FUSEREF) {
+        if (threadIdx.x < kMaxK) s_alpha[threadIdx.x] = ((int)threadIdx.x < a.hist_k) ? a.alpha[threadIdx.x] : 0.0f;
+        __syncthreads();
+    }
+    const int lane = threadIdx.x & 31;
+    const uint64_t warps_per_cta = kCodecThreads / 32;
+    const uint64_t nwarps = (uint64_t)gridDim.x * warps_per_cta;
+    const uint64_t gwarp = (uint64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
+    const uint64_t nfull = a.d / kTile;
+    for (uint64_t T = a.tile_begin + gwarp; T < nfull; T += nwarps) encode_tile<CODEC, NORM, SCALE, PHASE, true, FUSEREF>(a, s_alpha, T, lane);
+    if (nfull < a.ntile && gwarp == nfull % nwarps) encode_tile<CODEC, NORM, SCALE, PHASE, false, FUSEREF>(a, s_alpha, nfull, lane);
+}
+
+// ---------------------------------------------------------------------------
+// Encode fed by the bulk-copy pipeline (one scale per tile, full tiles only).
+// Virtual row list: the rows that make the reference (the k history rows when the
+// reference is combined here, else the reference itself, else nothing), then the M
+// gradient rows.  A chunk of 1024 coordinates = 8 tiles; two warps share a tile and
+// split its workers by parity, so 16 compute warps are busy per CTA.  Both warps of a
+// pair form the reference (the even one stores it).  Everything a warp computes is
+// what encode_tile computes; only where the operands come from differs.
+// ---------------------------------------------------------------------------
+constexpr int kEncPipeWarps = 16;
+constexpr int kEncPipeThreads = kEncPipeWarps * 32 + 32;   // + the producer warp
+
+struct EncodePipeArgs {
+    EncodeArgs e;
+    PipeRows rows;
+    int n_pre;          // rows ahead of the gradient rows
+};
+
+template <int CODEC, int NORM, int SCALE, bool FUSEREF>
+__global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const EncodePipeArgs pa) {
+    extern __shared__ unsigned char dyn_smem[];
+    __shared__ float s_alpha[kMaxK];
+    const EncodeArgs& a = pa.e;
+    if (FUSEREF && threadIdx.x < kMaxK) s_alpha[threadIdx.x] = ((int)threadIdx.x < a.hist_k) ? a.alpha[threadIdx.x] : 0.0f;
+    const PipeSmem pipe = pipe_setup(dyn_smem, kEncPipeWarps);   // ends with __syncthreads
+    const uint64_t nchunks = a.tile_begin / (kChunk / kTile);    // the chunks ahead of the directly read tiles
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == kEncPipeWarps) {
+        if (lane == 0) {
+            const uint32_t err = pipe_produce(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
+            if (err != kPipeOk) atomicMax(a.pipe_error, err);
+        }
+        return;
+    }
+    const uint32_t tile_in_chunk = (uint32_t)warp >> 1, half = (uint32_t)warp & 1u;
+    const uint32_t my = tile_in_chunk * (kTile * 4u) + (uint32_t)lane * 16u;   // byte offset inside a row chunk
+    const int nrows = pa.rows.nrows, n_pre = pa.n_pre;
+    uint32_t it = 0;
+    for (uint64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        const uint64_t T = c * (kChunk / kTile) + tile_in_chunk;
+        const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
+        const uint64_t q = T * 32u + (uint32_t)lane;
+        const uint32_t q_lo = (uint32_t)q, q_hi = (uint32_t)(q >> 32);
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f), op = r;
+        bool have_op = (NORM == TNG_NORM_NONE);
+        uint32_t rmax = 0;
+        for (int r0 = 0; r0 < nrows; r0 += kStageRows) {
+            const int n = (nrows - r0 < kStageRows) ? nrows - r0 : kStageRows;
+            const uint32_t s = it % kStages, use = it / kStages;
+            if (!__all_sync(kFullMask, mbar_wait(pipe.full[s], use & 1u))) {   // warp-uniform outcome
+                atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
+                return;
+            }
+            const uint32_t base = pipe.data + s * kStageBytes + my;
+            int ri = 0;
+            // rows that make the reference
+            for (; ri < n && r0 + ri < n_pre; ++ri) {
+                const float4 x = lds128(base + (uint32_t)ri * kRowBytes);
+                if (FUSEREF) {
+                    const float al = s_alpha[r0 + ri];
+                    r.x = __fmaf_rn(al, x.x, r.x); r.y = __fmaf_rn(al, x.y, r.y);
+                    r.z = __fmaf_rn(al, x.z, r.z); r.w = __fmaf_rn(al, x.w, r.w);
+                } else {
+                    r = x;
+                }
+            }
+            if (ri < n && !have_op) {   // the first gradient row is here: the reference is complete
+                if (FUSEREF && half == 0) *reinterpret_cast<float4*>(a.ref_out + i0) = r;
+                if (NORM == TNG_NORM_DIFF) {
+                    op = r;
+                } else {
+                    const float4 den = quot_den4(r, a.quot_eps);
+                    op = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z),
+                                     __fdiv_rn(1.0f, den.w));
+                }
+                have_op = true;
+            }
+            // this warp's workers among the gradient rows of the fill: m = half (mod 2), two at a time
+            int m = r0 + ri - n_pre;                       // worker of stage row ri
+            if (((uint32_t)m & 1u) != half) { ++m; ++ri; }
+            for (; ri + 2 < n; ri += 4, m += 4) {
+                const float4 g0 = lds128(base + (uint32_t)ri * kRowBytes);
+                const float4 g1 = lds128(base + (uint32_t)(ri + 2) * kRowBytes);
+                const uint32_t b0 = encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g0, op, (uint32_t)m, T, q_lo, q_hi, T, lane, 0xFu);
+                const uint32_t b1 = encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g1, op, (uint32_t)m + 2u, T, q_lo, q_hi, T, lane, 0xFu);
+                rmax = max(rmax, max(b0, b1));
+            }
+            if (ri < n) {
+                const float4 g0 = lds128(base + (uint32_t)ri * kRowBytes);
+                rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g0, op, (uint32_t)m, T, q_lo, q_hi, T, lane, 0xFu));
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pipe.empty[s]);   // this warp has read the stage
+            ++it;
+        }
+        // NaN or +inf scales are rare: only then count them, from the scales this warp wrote
+        if (rmax >= 0x7f800000u && lane == 0) {
+            unsigned long long bad = 0;
+            for (uint32_t m = half; m < a.M; m += 2) bad += (__float_as_uint(a.scales[(uint64_t)m * a.nblk + T]) >= 0x7f800000u) ? 1ull : 0ull;
+            atomicAdd(a.nonfinite, bad);
         }
     }
 }
@@ -190,126 +394,248 @@ struct DecodeArgs {
     const float* ref;
     float* out_a;
     float* out_b;
-    uint64_t d, ntile, nblk, block, wpw;
+    uint64_t d, ntile, block;
+    uint32_t nblk, wpw;
     uint32_t M;
+    uint32_t one;  // 1 as a run-time value: "w << s" is taken as w * (one << s), on the multiplier pipe
     int levels;
     float quot_eps;
+    float inv_m;   // 1/M when M is a power of two (then x * inv_m == x / M exactly), else 0
 };
 
+// Adds worker m's decoded values of the lane's four coordinates to acc.  `w` are the
+// tile's code words (the same in every lane); multiplying a word by pw = 2^(31-lane)
+// moves the lane's bit to the sign position.  A scale that is zero, NaN or infinite
+// decodes to +0 whatever the symbols say.
 template <int CODEC>
 __device__ __forceinline__ void decode_worker(const uint32_t (&w)[4 * CODEC], const float R, const int levels,
-                                              const int lane, const bool first, float (&acc)[4]) {
+                                              const uint32_t pw, const int lane, float (&acc)[4]) {
     const bool ok = !scale_is_bad(R);
-    float step = 0.f;
-    if (CODEC == TNG_CODEC_QSGD4) step = __fdiv_rn(R, (float)levels);
+    const uint32_t Re = ok ? __float_as_uint(R) : 0u;
+    const uint32_t okm = ok ? 0x80000000u : 0u;
+    if (CODEC == TNG_CODEC_TERN2) {
 #pragma unroll
-    for (int c = 0; c < 4; ++c) {
-        float vh;
-        if (CODEC == TNG_CODEC_TERN2) {
-            const uint32_t nz = (w[c * 2] >> lane) & 1u, neg = (w[c * 2 + 1] >> lane) & 1u;
-            vh = nz ? (neg ? -R : R) : 0.0f;
-        } else if (CODEC == TNG_CODEC_SIGN1) {
-            vh = ((w[c] >> lane) & 1u) ? R : -R;
-        } else {
+        for (int c = 0; c < 4; ++c) {
+            // sign plane -> sign bit of R; the add is skipped for the zero symbol (acc + 0 == acc)
+            const float sR = __uint_as_float(((w[c * 2 + 1] * pw) & okm) ^ Re);
+            if ((int)(w[c * 2] * pw) < 0) acc[c] = __fadd_rn(acc[c], sR);
+        }
+    } else if (CODEC == TNG_CODEC_SIGN1) {
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            const float sR = __uint_as_float((~(w[c] * pw) & okm) ^ Re);   // plus bit clear -> -R
+            acc[c] = __fadd_rn(acc[c], sR);
+        }
+    } else {
+        const float step = __fdiv_rn(R, (float)levels);
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
             const uint32_t L = ((w[c * 4] >> lane) & 1u) | (((w[c * 4 + 1] >> lane) & 1u) << 1) |
                                (((w[c * 4 + 2] >> lane) & 1u) << 2);
             const float mag = __fmul_rn((float)L, step);
-            vh = ((w[c * 4 + 3] >> lane) & 1u) ? -mag : mag;
+            const float vh = ok ? __uint_as_float(__float_as_uint(mag) ^ ((w[c * 4 + 3] * pw) & 0x80000000u)) : 0.0f;
+            acc[c] = __fadd_rn(acc[c], vh);
         }
-        if (!ok) vh = 0.0f;
-        acc[c] = first ? vh : __fadd_rn(acc[c], vh);
     }
 }
 
-template <int CODEC, int NORM>
-__global__ void __launch_bounds__(256) decode_kernel(const DecodeArgs a) {
-    const int lane = threadIdx.x & 31;
-    const uint64_t warps_per_cta = blockDim.x >> 5;
-    const uint64_t nwarps = (uint64_t)gridDim.x * warps_per_cta;
+template <int CODEC, int N>
+__device__ __forceinline__ void decode_batch(const DecodeArgs& a, const uint32_t* cp, const float* sp, const uint32_t m0,
+                                             const uint32_t pw, const int lane, float (&acc)[4]) {
     constexpr int kWords = 4 * CODEC;
-    for (uint64_t T = (uint64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5); T < a.ntile; T += nwarps) {
-        const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
-        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (NORM != TNG_NORM_NONE && a.ref) r = load4(a.ref, i0, a.d);
-        float4 den = make_float4(1.f, 1.f, 1.f, 1.f);
-        if (NORM == TNG_NORM_QUOT) den = quot_den4(r, a.quot_eps);
-        const uint64_t blk = (T * kTile) / a.block;
-        float acc[4] = {0.f, 0.f, 0.f, 0.f};
-        for (uint32_t m0 = 0; m0 < a.M; m0 += 2) {
-            uint32_t w[2][kWords];
-            float R[2];
+    uint4 wv[N][CODEC];
+    float R[N];
 #pragma unroll
-            for (int k = 0; k < 2; ++k) {
-                if (m0 + k < a.M) {
-                    const uint4* wp = reinterpret_cast<const uint4*>(a.codes + (uint64_t)(m0 + k) * a.wpw + T * kWords);
+    for (int k = 0; k < N; ++k) {
+        const uint4* wp = reinterpret_cast<const uint4*>(cp + (uint64_t)(m0 + k) * a.wpw);
 #pragma unroll
-                    for (int q = 0; q < CODEC; ++q) {
-                        const uint4 t = __ldg(wp + q);
-                        w[k][4 * q + 0] = t.x; w[k][4 * q + 1] = t.y; w[k][4 * q + 2] = t.z; w[k][4 * q + 3] = t.w;
-                    }
-                    R[k] = __ldg(a.scales + (uint64_t)(m0 + k) * a.nblk + blk);
-                }
-            }
+        for (int q = 0; q < CODEC; ++q) wv[k][q] = __ldcs(wp + q);
+        R[k] = __ldcs(sp + (uint64_t)(m0 + k) * a.nblk);
+    }
 #pragma unroll
-            for (int k = 0; k < 2; ++k)
-                if (m0 + k < a.M) decode_worker<CODEC>(w[k], R[k], a.levels, lane, (m0 + k) == 0, acc);
+    for (int k = 0; k < N; ++k) {
+        uint32_t w[kWords];
+#pragma unroll
+        for (int q = 0; q < CODEC; ++q) {
+            w[4 * q + 0] = wv[k][q].x; w[4 * q + 1] = wv[k][q].y; w[4 * q + 2] = wv[k][q].z; w[4 * q + 3] = wv[k][q].w;
         }
-        // average over the M workers (Algorithm 1), then put the reference back (Eq. 2 / Eq. 3)
+        decode_worker<CODEC>(w, R[k], a.levels, pw, lane, acc);
+    }
+}
+
+template <int CODEC, int NORM, bool FULL>
+__device__ __forceinline__ void decode_tile(const DecodeArgs& a, const uint64_t T, const int lane) {
+    constexpr int kWords = 4 * CODEC;
+    constexpr int kBatch = (CODEC == TNG_CODEC_QSGD4) ? 2 : 4;   // workers whose code words are in flight together
+    const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
+    const uint32_t pw = a.one << (31 - lane);
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (NORM != TNG_NORM_NONE && a.ref) r = FULL ? *reinterpret_cast<const float4*>(a.ref + i0) : load4(a.ref, i0, a.d);
+    float4 den = make_float4(1.f, 1.f, 1.f, 1.f);
+    if (NORM == TNG_NORM_QUOT) den = quot_den4(r, a.quot_eps);
+    const uint64_t blk = (a.block == (uint64_t)kTile) ? T : (T * kTile) / a.block;
+    // the sum starts from -0 so that (-0) + x == x bit for bit; the ternary path starts from +0
+    // because it skips zero symbols and +0 is what the sum of skipped terms is
+    const float z = (CODEC == TNG_CODEC_TERN2) ? 0.0f : -0.0f;
+    float acc[4] = {z, z, z, z};
+    const uint32_t* cp = a.codes + T * (uint64_t)kWords;
+    const float* sp = a.scales + blk;
+    const uint32_t m_batched = a.M - a.M % kBatch;
+    for (uint32_t m0 = 0; m0 < m_batched; m0 += kBatch) decode_batch<CODEC, kBatch>(a, cp, sp, m0, pw, lane, acc);
+    for (uint32_t m = m_batched; m < a.M; ++m) decode_batch<CODEC, 1>(a, cp, sp, m, pw, lane, acc);
+    // average over the M workers (Algorithm 1), then put the reference back (Eq. 2 / Eq. 3)
+    float4 o;
+    if (a.inv_m > 0.0f) {
+        o.x = __fmul_rn(acc[0], a.inv_m); o.y = __fmul_rn(acc[1], a.inv_m); o.z = __fmul_rn(acc[2], a.inv_m); o.w = __fmul_rn(acc[3], a.inv_m);
+    } else {
         const float fm = (float)a.M;
-        float4 o;
         o.x = __fdiv_rn(acc[0], fm); o.y = __fdiv_rn(acc[1], fm); o.z = __fdiv_rn(acc[2], fm); o.w = __fdiv_rn(acc[3], fm);
-        if (NORM == TNG_NORM_DIFF) {
-            o.x = __fadd_rn(r.x, o.x); o.y = __fadd_rn(r.y, o.y); o.z = __fadd_rn(r.z, o.z); o.w = __fadd_rn(r.w, o.w);
-        } else if (NORM == TNG_NORM_QUOT) {
-            o.x = __fmul_rn(den.x, o.x); o.y = __fmul_rn(den.y, o.y); o.z = __fmul_rn(den.z, o.z); o.w = __fmul_rn(den.w, o.w);
-        }
+    }
+    if (NORM == TNG_NORM_DIFF) {
+        o.x = __fadd_rn(r.x, o.x); o.y = __fadd_rn(r.y, o.y); o.z = __fadd_rn(r.z, o.z); o.w = __fadd_rn(r.w, o.w);
+    } else if (NORM == TNG_NORM_QUOT) {
+        o.x = __fmul_rn(den.x, o.x); o.y = __fmul_rn(den.y, o.y); o.z = __fmul_rn(den.z, o.z); o.w = __fmul_rn(den.w, o.w);
+    }
+    if (FULL) {
+        if (a.out_a) *reinterpret_cast<float4*>(a.out_a + i0) = o;
+        if (a.out_b) *reinterpret_cast<float4*>(a.out_b + i0) = o;
+    } else {
         if (a.out_a) store4(a.out_a, i0, a.d, o);
         if (a.out_b) store4(a.out_b, i0, a.d, o);
     }
 }
 
-int grid_for_tiles(uint64_t ntile, int sm_count, int ctas_per_sm) {
+template <int CODEC, int NORM>
+__global__ void __launch_bounds__(kCodecThreads, 3) decode_kernel(const DecodeArgs a) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t warps_per_cta = kCodecThreads / 32;
+    const uint64_t nwarps = (uint64_t)gridDim.x * warps_per_cta;
+    const uint64_t gwarp = (uint64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
+    const uint64_t nfull = a.d / kTile;
+    for (uint64_t T = gwarp; T < nfull; T += nwarps) decode_tile<CODEC, NORM, true>(a, T, lane);
+    if (nfull < a.ntile && gwarp == nfull % nwarps) decode_tile<CODEC, NORM, false>(a, nfull, lane);
+}
+
+// Persistent launch: as many CTAs as fit on the GPU at once (occupancy of this very
+// instantiation times the SM count), fewer when there are not enough tiles.
+template <typename Kern>
+int persistent_grid(Kern kern, uint64_t ntile, int sm_count) {
+    int per_sm = 0;
+    if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kern, kCodecThreads, 0) != cudaSuccess || per_sm < 1) {
+        (void)cudaGetLastError();
+        per_sm = 1;
+    }
     const uint64_t want = (ntile + 7) / 8;   // 8 warps per CTA, one tile per warp per pass
-    const uint64_t cap = (uint64_t)sm_count * ctas_per_sm;
+    const uint64_t cap = (uint64_t)sm_count * (uint64_t)per_sm;
     return (int)(want < cap ? (want ? want : 1) : cap);
 }
 
-template <int CODEC, int NORM, int SCALE>
-cudaError_t encode_dispatch_phase(const EncodeArgs& a, int phase, int grid, cudaStream_t st) {
-    if (phase == kPhaseFused) encode_kernel<CODEC, NORM, SCALE, kPhaseFused><<<grid, 256, 0, st>>>(a);
-    else if (phase == kPhaseStat) encode_kernel<CODEC, NORM, SCALE, kPhaseStat><<<grid, 256, 0, st>>>(a);
-    else encode_kernel<CODEC, NORM, SCALE, kPhaseQuant><<<grid, 256, 0, st>>>(a);
+template <int CODEC, int NORM, int SCALE, int PHASE, bool FUSEREF>
+cudaError_t encode_launch_direct(const EncodeArgs& a, int sm_count, cudaStream_t st) {
+    static int per_tiles_grid = 0;   // grid when tiles are plentiful
+    auto kern = encode_kernel<CODEC, NORM, SCALE, PHASE, FUSEREF>;
+    if (per_tiles_grid == 0) per_tiles_grid = persistent_grid(kern, ~0ull >> 8, sm_count);
+    const uint64_t want = (a.ntile - a.tile_begin + 7) / 8;
+    const int grid = (int)(want < (uint64_t)per_tiles_grid ? (want ? want : 1) : (uint64_t)per_tiles_grid);
+    kern<<<grid, kCodecThreads, 0, st>>>(a);
     return cudaGetLastError();
 }
+
+constexpr uint64_t kEncPipeMinChunks = 16;   // shorter vectors take the direct kernel
+
+// One scale per tile: the whole chunks go through the staged kernel, the remaining tiles
+// (fewer than 8 full ones and a ragged one) through the direct kernel.
+template <int CODEC, int NORM, int SCALE, bool FUSEREF>
+cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t st, int* launches) {
+    const uint64_t nchunks = a0.d / kChunk;
+    EncodeArgs a = a0;
+    a.tile_begin = 0;
+    if (nchunks >= kEncPipeMinChunks) {
+        static bool configured = false;   // opt in to the large dynamic shared memory once per instantiation
+        auto kern = encode_pipe_kernel<CODEC, NORM, SCALE, FUSEREF>;
+        if (!configured) {
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
+            if (e != cudaSuccess) return e;
+            configured = true;
+        }
+        EncodePipeArgs pa;
+        pa.e = a;
+        pa.e.tile_begin = nchunks * (kChunk / kTile);
+        pa.rows.nrows = 0;
+        if (FUSEREF) {
+            for (int j = 0; j < a.hist_k; ++j) pa.rows.row[pa.rows.nrows++] = a.hist[j];
+        } else if (NORM != TNG_NORM_NONE && a.ref) {
+            pa.rows.row[pa.rows.nrows++] = a.ref;
+        }
+        pa.n_pre = pa.rows.nrows;
+        for (uint32_t m = 0; m < a.M; ++m) pa.rows.row[pa.rows.nrows++] = a.grads + (uint64_t)m * a.ld;
+        const int grid = (int)(nchunks < (uint64_t)sm_count ? nchunks : (uint64_t)sm_count);
+        kern<<<grid, kEncPipeThreads, kPipeSmemBytes, st>>>(pa);
+        ++*launches;
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        a.tile_begin = pa.e.tile_begin;
+        if (a.tile_begin >= a.ntile) return cudaSuccess;
+    }
+    ++*launches;
+    return encode_launch_direct<CODEC, NORM, SCALE, kPhaseFused, FUSEREF>(a, sm_count, st);
+}
+
+template <int CODEC, int NORM, int SCALE, int PHASE>
+cudaError_t encode_launch(const EncodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
+    if (PHASE == kPhaseFused) {
+        if (NORM != TNG_NORM_NONE && a.hist_k > 0)
+            return encode_launch_tiles<CODEC, NORM, SCALE, (NORM != TNG_NORM_NONE)>(a, sm_count, st, launches);
+        return encode_launch_tiles<CODEC, NORM, SCALE, false>(a, sm_count, st, launches);
+    }
+    ++*launches;
+    return encode_launch_direct<CODEC, NORM, SCALE, PHASE, false>(a, sm_count, st);
+}
+template <int CODEC, int NORM, int SCALE>
+cudaError_t encode_dispatch_phase(const EncodeArgs& a, int phase, int sm_count, cudaStream_t st, int* launches) {
+    if (phase == kPhaseFused) return encode_launch<CODEC, NORM, SCALE, kPhaseFused>(a, sm_count, st, launches);
+    if (phase == kPhaseStat) return encode_launch<CODEC, NORM, SCALE, kPhaseStat>(a, sm_count, st, launches);
+    return encode_launch<CODEC, NORM, SCALE, kPhaseQuant>(a, sm_count, st, launches);
+}
 template <int CODEC, int NORM>
-cudaError_t encode_dispatch_scale(const EncodeArgs& a, int scale, int phase, int grid, cudaStream_t st) {
-    return scale == 0 ? encode_dispatch_phase<CODEC, NORM, 0>(a, phase, grid, st)
-                      : encode_dispatch_phase<CODEC, NORM, 1>(a, phase, grid, st);
+cudaError_t encode_dispatch_scale(const EncodeArgs& a, int scale, int phase, int sm_count, cudaStream_t st, int* launches) {
+    return scale == 0 ? encode_dispatch_phase<CODEC, NORM, 0>(a, phase, sm_count, st, launches)
+                      : encode_dispatch_phase<CODEC, NORM, 1>(a, phase, sm_count, st, launches);
 }
 template <int CODEC>
-cudaError_t encode_dispatch_norm(const EncodeArgs& a, int norm, int scale, int phase, int grid, cudaStream_t st) {
+cudaError_t encode_dispatch_norm(const EncodeArgs& a, int norm, int scale, int phase, int sm_count, cudaStream_t st, int* launches) {
     switch (norm) {
-        case TNG_NORM_DIFF: return encode_dispatch_scale<CODEC, TNG_NORM_DIFF>(a, scale, phase, grid, st);
-        case TNG_NORM_QUOT: return encode_dispatch_scale<CODEC, TNG_NORM_QUOT>(a, scale, phase, grid, st);
-        default: return encode_dispatch_scale<CODEC, TNG_NORM_NONE>(a, scale, phase, grid, st);
+        case TNG_NORM_DIFF: return encode_dispatch_scale<CODEC, TNG_NORM_DIFF>(a, scale, phase, sm_count, st, launches);
+        case TNG_NORM_QUOT: return encode_dispatch_scale<CODEC, TNG_NORM_QUOT>(a, scale, phase, sm_count, st, launches);
+        default: return encode_dispatch_scale<CODEC, TNG_NORM_NONE>(a, scale, phase, sm_count, st, launches);
     }
 }
-cudaError_t encode_dispatch(const EncodeArgs& a, int codec, int norm, int scale, int phase, int grid, cudaStream_t st) {
+cudaError_t encode_dispatch(const EncodeArgs& a, int codec, int norm, int scale, int phase, int sm_count, cudaStream_t st,
+                            int* launches) {
     switch (codec) {
-        case TNG_CODEC_SIGN1: return encode_dispatch_norm<TNG_CODEC_SIGN1>(a, norm, scale, phase, grid, st);
-        case TNG_CODEC_TERN2: return encode_dispatch_norm<TNG_CODEC_TERN2>(a, norm, scale, phase, grid, st);
-        default: return encode_dispatch_norm<TNG_CODEC_QSGD4>(a, norm, scale, phase, grid, st);
+        case TNG_CODEC_SIGN1: return encode_dispatch_norm<TNG_CODEC_SIGN1>(a, norm, scale, phase, sm_count, st, launches);
+        case TNG_CODEC_TERN2: return encode_dispatch_norm<TNG_CODEC_TERN2>(a, norm, scale, phase, sm_count, st, launches);
+        default: return encode_dispatch_norm<TNG_CODEC_QSGD4>(a, norm, scale, phase, sm_count, st, launches);
     }
 }
 
-template <int CODEC>
-cudaError_t decode_dispatch_norm(const DecodeArgs& a, int norm, int grid, cudaStream_t st) {
-    switch (norm) {
-        case TNG_NORM_DIFF: decode_kernel<CODEC, TNG_NORM_DIFF><<<grid, 256, 0, st>>>(a); break;
-        case TNG_NORM_QUOT: decode_kernel<CODEC, TNG_NORM_QUOT><<<grid, 256, 0, st>>>(a); break;
-        default: decode_kernel<CODEC, TNG_NORM_NONE><<<grid, 256, 0, st>>>(a); break;
-    }
+template <int CODEC, int NORM>
+cudaError_t decode_launch(const DecodeArgs& a, int sm_count, cudaStream_t st) {
+    static int per_tiles_grid = 0;
+    auto kern = decode_kernel<CODEC, NORM>;
+    if (per_tiles_grid == 0) per_tiles_grid = persistent_grid(kern, ~0ull >> 8, sm_count);
+    const uint64_t want = (a.ntile + 7) / 8;
+    const int grid = (int)(want < (uint64_t)per_tiles_grid ? (want ? want : 1) : (uint64_t)per_tiles_grid);
+    kern<<<grid, kCodecThreads, 0, st>>>(a);
     return cudaGetLastError();
+}
+template <int CODEC>
+cudaError_t decode_dispatch_norm(const DecodeArgs& a, int norm, int sm_count, cudaStream_t st) {
+    switch (norm) {
+        case TNG_NORM_DIFF: return decode_launch<CODEC, TNG_NORM_DIFF>(a, sm_count, st);
+        case TNG_NORM_QUOT: return decode_launch<CODEC, TNG_NORM_QUOT>(a, sm_count, st);
+        default: return decode_launch<CODEC, TNG_NORM_NONE>(a, sm_count, st);
+    }
 }
 
 }  // namespace
@@ -322,25 +648,28 @@ size_t tree_tmp_floats(const CodecGeom& g) {
     return (size_t)(2 * (uint64_t)g.M * g.nblk * chunks);
 }
 
-cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref, uint32_t step,
-                          uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp, FuseBlock* fb,
+bool encode_can_fuse_reference(const CodecGeom& g) { return g.block == kTile && g.norm != TNG_NORM_NONE; }
+
+cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref, const RefFusion* fusion,
+                          uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp, FuseBlock* fb,
                           int sm_count, cudaStream_t st, int* launches) {
     EncodeArgs a;
-    a.grads = grads; a.ref = ref; a.codes = codes; a.scales = scales; a.tile_stat = tile_stat;
-    a.nonfinite = &fb->nonfinite;
-    a.ld = ld; a.d = g.d; a.ntile = g.ntile; a.nblk = g.nblk; a.block = g.block; a.wpw = g.wpw;
-    a.M = g.M; a.step = step; a.seed_lo = g.seed_lo; a.seed_hi = g.seed_hi; a.levels = g.levels;
-    a.quot_eps = g.quot_eps;
-    const int grid = grid_for_tiles(g.ntile, sm_count, 8);
-    cudaError_t e;
-    if (g.block == kTile) {
-        e = encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseFused, grid, st);
-        ++*launches;
-        return e;
+    a.hist_k = 0; a.alpha = nullptr; a.ref_out = nullptr;
+    for (int j = 0; j < kMaxK; ++j) a.hist[j] = nullptr;
+    if (fusion && fusion->k > 0 && encode_can_fuse_reference(g)) {
+        a.hist_k = fusion->k; a.alpha = fusion->alpha; a.ref_out = fusion->ref_out;
+        for (int j = 0; j < fusion->k; ++j) a.hist[j] = fusion->rows[j];
     }
+    a.grads = grads; a.ref = ref; a.codes = codes; a.scales = scales; a.tile_stat = tile_stat;
+    a.nonfinite = &fb->nonfinite; a.pipe_error = &fb->pipe_error; a.tile_begin = 0;
+    a.ld = (uint32_t)ld; a.d = g.d; a.ntile = g.ntile; a.nblk = (uint32_t)g.nblk; a.block = g.block; a.wpw = (uint32_t)g.wpw;
+    a.M = g.M; a.step = step; a.levels = g.levels; a.pow24 = 1u << 24;
+    a.quot_eps = g.quot_eps;
+    philox_round_keys(g.seed_lo, g.seed_hi, a.rk);
+    cudaError_t e;
+    if (g.block == kTile) return encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseFused, sm_count, st, launches);
     // general block size: per-tile statistic -> per-block tree -> quantise
-    e = encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseStat, grid, st);
-    ++*launches;
+    e = encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseStat, sm_count, st, launches);
     if (e != cudaSuccess) return e;
     const float* in = tile_stat;
     uint64_t n_in = g.ntile;
@@ -364,23 +693,21 @@ cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, c
         float* t = ping; ping = pong; pong = t;
     }
     if (e != cudaSuccess) return e;
-    e = encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseQuant, grid, st);
-    ++*launches;
-    return e;
+    return encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseQuant, sm_count, st, launches);
 }
 
 cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref,
                           float* out_a, float* out_b, int sm_count, cudaStream_t st, int* launches) {
     DecodeArgs a;
     a.codes = codes; a.scales = scales; a.ref = ref; a.out_a = out_a; a.out_b = out_b;
-    a.d = g.d; a.ntile = g.ntile; a.nblk = g.nblk; a.block = g.block; a.wpw = g.wpw; a.M = g.M;
-    a.levels = g.levels; a.quot_eps = g.quot_eps;
-    const int grid = grid_for_tiles(g.ntile, sm_count, 8);
+    a.d = g.d; a.ntile = g.ntile; a.nblk = (uint32_t)g.nblk; a.block = g.block; a.wpw = (uint32_t)g.wpw; a.M = g.M;
+    a.one = 1u; a.levels = g.levels; a.quot_eps = g.quot_eps;
+    a.inv_m = ((g.M & (g.M - 1)) == 0) ? 1.0f / (float)g.M : 0.0f;
     cudaError_t e;
     switch (g.codec) {
-        case TNG_CODEC_SIGN1: e = decode_dispatch_norm<TNG_CODEC_SIGN1>(a, g.norm, grid, st); break;
-        case TNG_CODEC_TERN2: e = decode_dispatch_norm<TNG_CODEC_TERN2>(a, g.norm, grid, st); break;
-        default: e = decode_dispatch_norm<TNG_CODEC_QSGD4>(a, g.norm, grid, st); break;
+        case TNG_CODEC_SIGN1: e = decode_dispatch_norm<TNG_CODEC_SIGN1>(a, g.norm, sm_count, st); break;
+        case TNG_CODEC_TERN2: e = decode_dispatch_norm<TNG_CODEC_TERN2>(a, g.norm, sm_count, st); break;
+        default: e = decode_dispatch_norm<TNG_CODEC_QSGD4>(a, g.norm, sm_count, st); break;
     }
     ++*launches;
     return e;

@@ -15,24 +15,34 @@ constexpr unsigned kFullMask = 0xFFFFFFFFu;
 
 // ---------------------------------------------------------------------------
 // Philox4x32-10 (Salmon, Moraes, Dror, Shaw, SC'11).  One call yields the four
-// uniforms of the four coordinates a lane owns.
+// uniforms of the four coordinates a lane owns.  The ten round keys (key plus
+// multiples of the Weyl constants) are the same for every call of a launch, so
+// the host computes them once and the kernel reads them from its arguments.
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ uint4 philox4x32_10(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
-                                               uint32_t k0, uint32_t k1) {
-    constexpr uint32_t kMul0 = 0xD2511F53u, kMul1 = 0xCD9E8D57u;
-    constexpr uint32_t kWeyl0 = 0x9E3779B9u, kWeyl1 = 0xBB67AE85u;
+constexpr uint32_t kPhiloxMul0 = 0xD2511F53u, kPhiloxMul1 = 0xCD9E8D57u;
+constexpr uint32_t kPhiloxWeyl0 = 0x9E3779B9u, kPhiloxWeyl1 = 0xBB67AE85u;
+
+inline void philox_round_keys(uint32_t k0, uint32_t k1, uint32_t (&rk)[20]) {
+    for (int round = 0; round < 10; ++round) {
+        rk[2 * round] = k0;
+        rk[2 * round + 1] = k1;
+        k0 += kPhiloxWeyl0;
+        k1 += kPhiloxWeyl1;
+    }
+}
+
+__device__ __forceinline__ uint4 philox4x32_10_rk(uint32_t c0, uint32_t c1, uint32_t c2, uint32_t c3,
+                                                  const uint32_t (&rk)[20]) {
 #pragma unroll
     for (int round = 0; round < 10; ++round) {
-        const uint64_t p0 = static_cast<uint64_t>(kMul0) * c0;
-        const uint64_t p1 = static_cast<uint64_t>(kMul1) * c2;
-        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ k0;
-        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ k1;
+        const uint64_t p0 = static_cast<uint64_t>(kPhiloxMul0) * c0;
+        const uint64_t p1 = static_cast<uint64_t>(kPhiloxMul1) * c2;
+        const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ c1 ^ rk[2 * round];
+        const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ c3 ^ rk[2 * round + 1];
         c1 = static_cast<uint32_t>(p1);
         c3 = static_cast<uint32_t>(p0);
         c0 = n0;
         c2 = n2;
-        k0 += kWeyl0;
-        k1 += kWeyl1;
     }
     return make_uint4(c0, c1, c2, c3);
 }

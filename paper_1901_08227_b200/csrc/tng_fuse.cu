@@ -12,6 +12,7 @@
 // (an arrival counter, nobody waits), which keeps the sums run-to-run identical.
 #include "tng_device.cuh"
 #include "tng_internal.h"
+#include "tng_pipeline.cuh"
 
 namespace tng {
 
@@ -35,6 +36,164 @@ struct DotsShape {
     static constexpr int kPairs = SAME ? NA * (NA + 1) / 2 : NA * NB;
     static constexpr int kAcc = SAME ? kPairs + NA + 1 : kPairs;   // + rhs + grad_sq
 };
+
+// CTA reduction (lanes by butterfly, warps in warp order), one partial row per CTA, and
+// the CTA that arrives last adds the partial rows in CTA order: run-to-run identical sums,
+// nobody waits.  `tid` in [0, nthreads) indexes the threads that hold accumulators; every
+// thread of the CTA must call this (it contains __syncthreads), the others with tid >= nthreads.
+template <int kAcc, int kPairs, bool SAME>
+__device__ __forceinline__ void dots_finish(const double (&acc)[kAcc], const DotsArgs& a, const bool with_g, const int tid,
+                                            const int nthreads) {
+    __shared__ double warp_part[kDotsThreads / 32][kAcc];
+    __shared__ bool is_last;
+    const int lane = tid & 31, warp = tid >> 5;
+    if (tid < nthreads) {
+#pragma unroll
+        for (int i = 0; i < kAcc; ++i) {
+            double v = acc[i];
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(kFullMask, v, off);
+            if (lane == 0) warp_part[warp][i] = v;
+        }
+    }
+    __syncthreads();
+    if (tid < kAcc) {
+        double v = 0.0;
+        for (int w = 0; w < nthreads / 32; ++w) v += warp_part[w][tid];
+        a.partials[(uint64_t)blockIdx.x * kDotsMaxAcc + tid] = v;
+    }
+    __threadfence();
+    __syncthreads();
+    if (tid == 0) {
+        const uint32_t prev = atomicAdd(&a.fb->dots_arrivals, 1u);
+        is_last = (prev == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    if (tid < kAcc) {
+        double v = 0.0;
+        for (uint32_t b = 0; b < gridDim.x; ++b) v += __ldcg(a.partials + (uint64_t)b * kDotsMaxAcc + tid);
+        if (SAME && tid >= kPairs) v /= (double)a.M;   // rhs and grad_sq use the mean
+        if (!(SAME && !with_g && tid >= kPairs)) a.fb->gram[a.dst[tid]] = v;
+    }
+    if (tid == 0) a.fb->dots_arrivals = 0;   // ready for the next launch on this stream
+}
+
+// ---------------------------------------------------------------------------
+// Statistics pass fed by the bulk-copy pipeline (k <= 8 history rows in one launch).
+// Virtual row list: h_1..h_k, then g^0..g^{M-1}.  A chunk of 1024 coordinates of up to 16
+// rows is one stage; consumer thread t owns coordinates 4t..4t+3 of the chunk, keeps the
+// history values of the chunk in registers while the gradient rows stream through the
+// following fills, and accumulates exactly what dots_kernel accumulates.  The ragged end
+// of the vectors (d mod 1024) is read directly.
+// ---------------------------------------------------------------------------
+constexpr int kDotsPipeThreads = kDotsThreads + 32;   // 8 consumer warps + 1 producer warp
+constexpr uint64_t kDotsPipeMinCoords = 16 * kChunk;    // shorter vectors take the direct kernel
+
+struct DotsPipeArgs {
+    DotsArgs base;      // rows_a = history rows, grads/ld/M, partials, fb, dst
+    PipeRows rows;      // history rows then gradient rows
+};
+
+// acc += products of the four coordinates held in ha[] (history) and gs/gq (sum and sum of
+// squares of the gradients at these coordinates, fp32, m ascending)
+template <int NA>
+__device__ __forceinline__ void dots_accum4(const float4 (&ha)[NA], const float4 gs, const float4 gq, const bool with_g,
+                                            double (&acc)[NA * (NA + 1) / 2 + NA + 1]) {
+    constexpr int kPairs = NA * (NA + 1) / 2;
+#pragma unroll
+    for (int comp = 0; comp < 4; ++comp) {
+        double da[NA];
+#pragma unroll
+        for (int j = 0; j < NA; ++j) da[j] = (double)(comp == 0 ? ha[j].x : comp == 1 ? ha[j].y : comp == 2 ? ha[j].z : ha[j].w);
+        int p = 0;
+#pragma unroll
+        for (int i = 0; i < NA; ++i)
+#pragma unroll
+            for (int j = i; j < NA; ++j) { acc[p] = fma(da[i], da[j], acc[p]); ++p; }
+        if (with_g) {
+            const double dg = (double)(comp == 0 ? gs.x : comp == 1 ? gs.y : comp == 2 ? gs.z : gs.w);
+#pragma unroll
+            for (int i = 0; i < NA; ++i) acc[kPairs + i] = fma(da[i], dg, acc[kPairs + i]);
+            acc[kPairs + NA] += (double)(comp == 0 ? gq.x : comp == 1 ? gq.y : comp == 2 ? gq.z : gq.w);
+        }
+    }
+}
+
+__device__ __forceinline__ void grad_sums(float4& gs, float4& gq, const float4 g) {
+    gs.x += g.x; gs.y += g.y; gs.z += g.z; gs.w += g.w;
+    gq.x = fmaf(g.x, g.x, gq.x); gq.y = fmaf(g.y, g.y, gq.y); gq.z = fmaf(g.z, g.z, gq.z); gq.w = fmaf(g.w, g.w, gq.w);
+}
+
+template <int NA>
+__global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const DotsPipeArgs pa) {
+    extern __shared__ unsigned char dyn_smem[];
+    constexpr int kPairs = NA * (NA + 1) / 2;
+    constexpr int kAcc = kPairs + NA + 1;
+    const DotsArgs& a = pa.base;
+    const PipeSmem pipe = pipe_setup(dyn_smem, kDotsThreads / 32);
+    const bool with_g = a.grads != nullptr;
+    const uint64_t nchunks = a.d / kChunk;
+    const int tid = threadIdx.x;
+    double acc[kAcc];
+#pragma unroll
+    for (int i = 0; i < kAcc; ++i) acc[i] = 0.0;
+
+    if (tid >= kDotsThreads) {
+        // ---- producer warp: one thread feeds the stages
+        if (tid == kDotsThreads) {
+            const uint32_t err = pipe_produce(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
+            if (err != kPipeOk) atomicMax(&a.fb->pipe_error, err);
+        }
+    } else {
+        // ---- consumers
+        const int lane = tid & 31;
+        const uint32_t my = (uint32_t)tid * 16u;                  // byte offset of the thread's float4 inside a row chunk
+        const int nrows = pa.rows.nrows;
+        uint32_t it = 0;
+        bool alive = true;
+        for (uint64_t c = blockIdx.x; c < nchunks && alive; c += gridDim.x) {
+            float4 ha[NA];
+            float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), gq = make_float4(0.f, 0.f, 0.f, 0.f);
+            for (int r0 = 0; r0 < nrows; r0 += kStageRows) {
+                const int n = (nrows - r0 < kStageRows) ? nrows - r0 : kStageRows;
+                const uint32_t s = it % kStages, use = it / kStages;
+                if (!__all_sync(kFullMask, mbar_wait(pipe.full[s], use & 1u))) {   // warp-uniform outcome
+                    atomicMax(&a.fb->pipe_error, (uint32_t)kPipeFullTimeout);
+                    alive = false;
+                    break;
+                }
+                const uint32_t base = pipe.data + s * kStageBytes + my;
+                int r = 0;
+                if (r0 == 0) {
+#pragma unroll
+                    for (int j = 0; j < NA; ++j) ha[j] = lds128(base + (uint32_t)j * kRowBytes);
+                    r = NA;
+                }
+                for (; r < n; ++r) grad_sums(gs, gq, lds128(base + (uint32_t)r * kRowBytes));
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pipe.empty[s]);       // this warp has read the stage
+                ++it;
+            }
+            if (alive) dots_accum4<NA>(ha, gs, gq, with_g, acc);
+        }
+        // ---- ragged end: coordinates [nchunks*1024, d) straight from global memory
+        const uint64_t ngroups = (a.d + 3) / 4;
+        for (uint64_t grp = nchunks * (kChunk / 4) + (uint64_t)blockIdx.x * kDotsThreads + tid; grp < ngroups;
+             grp += (uint64_t)gridDim.x * kDotsThreads) {
+            const uint64_t i0 = grp * 4;
+            float4 ha[NA];
+#pragma unroll
+            for (int j = 0; j < NA; ++j) ha[j] = load4_stream(a.rows_a[j], i0, a.d);
+            float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), gq = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (with_g)
+                for (uint32_t m = 0; m < a.M; ++m) grad_sums(gs, gq, load4_stream(a.grads + (uint64_t)m * a.ld, i0, a.d));
+            dots_accum4<NA>(ha, gs, gq, with_g, acc);
+        }
+    }
+    dots_finish<kAcc, kPairs, true>(acc, a, with_g, tid, kDotsThreads);
+}
 
 template <int NA, int NB, bool SAME>
 __global__ void __launch_bounds__(kDotsThreads, 1) dots_kernel(const DotsArgs a) {
@@ -103,40 +262,7 @@ __global__ void __launch_bounds__(kDotsThreads, 1) dots_kernel(const DotsArgs a)
         }
     }
 
-    // ---- CTA reduction: lanes by butterfly, warps in warp order
-    __shared__ double warp_part[kDotsThreads / 32][kAcc];
-    __shared__ bool is_last;
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-#pragma unroll
-    for (int i = 0; i < kAcc; ++i) {
-        double v = acc[i];
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(kFullMask, v, off);
-        if (lane == 0) warp_part[warp][i] = v;
-    }
-    __syncthreads();
-    if (threadIdx.x < kAcc) {
-        double v = 0.0;
-        for (int w = 0; w < kDotsThreads / 32; ++w) v += warp_part[w][threadIdx.x];
-        a.partials[(uint64_t)blockIdx.x * kDotsMaxAcc + threadIdx.x] = v;
-    }
-    // ---- the CTA that arrives last adds the partials in CTA order
-    __threadfence();
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        const uint32_t prev = atomicAdd(&a.fb->dots_arrivals, 1u);
-        is_last = (prev == gridDim.x - 1);
-    }
-    __syncthreads();
-    if (!is_last) return;
-    __threadfence();
-    if (threadIdx.x < kAcc) {
-        double v = 0.0;
-        for (uint32_t b = 0; b < gridDim.x; ++b) v += __ldcg(a.partials + (uint64_t)b * kDotsMaxAcc + threadIdx.x);
-        if (SAME && threadIdx.x >= Shape::kPairs) v /= (double)a.M;   // rhs and grad_sq use the mean
-        if (!(SAME && !with_g && threadIdx.x >= Shape::kPairs)) a.fb->gram[a.dst[threadIdx.x]] = v;
-    }
-    if (threadIdx.x == 0) a.fb->dots_arrivals = 0;   // ready for the next launch on this stream
+    dots_finish<kAcc, Shape::kPairs, SAME>(acc, a, with_g, threadIdx.x, kDotsThreads);
 }
 
 template <int NA>
@@ -148,6 +274,30 @@ template <int NB>
 cudaError_t dots_cross(const DotsArgs& a, int grid, cudaStream_t st) {
     dots_kernel<8, NB, false><<<grid, kDotsThreads, 0, st>>>(a);
     return cudaGetLastError();
+}
+
+template <int NA>
+cudaError_t dots_pipe(const DotsPipeArgs& pa, int grid, cudaStream_t st) {
+    static bool configured = false;   // opt in to the large dynamic shared memory once per instantiation
+    if (!configured) {
+        cudaError_t e = cudaFuncSetAttribute(dots_pipe_kernel<NA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
+        if (e != cudaSuccess) return e;
+        configured = true;
+    }
+    dots_pipe_kernel<NA><<<grid, kDotsPipeThreads, kPipeSmemBytes, st>>>(pa);
+    return cudaGetLastError();
+}
+cudaError_t dots_pipe_n(int n, const DotsPipeArgs& pa, int grid, cudaStream_t st) {
+    switch (n) {
+        case 1: return dots_pipe<1>(pa, grid, st);
+        case 2: return dots_pipe<2>(pa, grid, st);
+        case 3: return dots_pipe<3>(pa, grid, st);
+        case 4: return dots_pipe<4>(pa, grid, st);
+        case 5: return dots_pipe<5>(pa, grid, st);
+        case 6: return dots_pipe<6>(pa, grid, st);
+        case 7: return dots_pipe<7>(pa, grid, st);
+        default: return dots_pipe<8>(pa, grid, st);
+    }
 }
 
 cudaError_t dots_same_n(int n, const DotsArgs& a, int grid, cudaStream_t st) {
@@ -329,6 +479,26 @@ cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float
     DotsArgs a;
     a.grads = grads; a.partials = partials; a.fb = fb; a.d = d; a.ld = ld; a.M = M;
     cudaError_t e = cudaSuccess;
+    // long vectors, at most 8 history rows: the staged kernel
+    if (k <= 8 && d >= kDotsPipeMinCoords) {
+        DotsPipeArgs pa;
+        for (int j = 0; j < 8; ++j) a.rows_a[j] = a.rows_b[j] = rows[j < k ? j : 0];
+        int p = 0;
+        for (int i = 0; i < k; ++i)
+            for (int j = i; j < k; ++j) a.dst[p++] = (short)(i * kGramStride + j);
+        for (int i = 0; i < k; ++i) a.dst[p++] = (short)(kGramRhs + i);
+        a.dst[p++] = (short)kGramGG;
+        pa.base = a;
+        pa.rows.nrows = 0;
+        for (int j = 0; j < k; ++j) pa.rows.row[pa.rows.nrows++] = rows[j];
+        if (grads)
+            for (uint32_t m = 0; m < M; ++m) pa.rows.row[pa.rows.nrows++] = grads + (uint64_t)m * ld;
+        const uint64_t nchunks = d / kChunk;
+        const int pgrid = (int)(nchunks < (uint64_t)sm_count ? nchunks : (uint64_t)sm_count);
+        e = dots_pipe_n(k, pa, pgrid, st);
+        ++*launches;
+        return e;
+    }
     // chunks of at most 8 history vectors: diagonal blocks (with rhs) and, for k > 8, the cross block
     for (int lo = 0; lo < k && e == cudaSuccess; lo += 8) {
         const int n = (k - lo < 8) ? k - lo : 8;

@@ -24,6 +24,8 @@ struct FuseBlock {
     float alpha32[kMaxK];
     uint32_t fallback;
     uint32_t dots_arrivals;          // CTAs that finished the current dots launch
+    uint32_t pipe_error;             // nonzero: a bounded wait of a staged kernel gave up (PipeError)
+    uint32_t pad_;
     unsigned long long nonfinite;    // NaN/Inf block scales seen so far
 };
 
@@ -54,8 +56,19 @@ cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const Fu
 // tile_stat: M*ntile floats, tree_tmp: scratch of tree_tmp_floats(geom) floats; both
 // only used when geom.block != 128.
 size_t tree_tmp_floats(const CodecGeom& g);
+// Optional: let the encode pass build the reference itself, r = sum_j alpha[j] rows[j] (the
+// combine step's fp32 fma chain), writing it to ref_out; saves one pass over the ring and
+// hides the encode arithmetic behind the ring's memory traffic.  Only for block == 128 with
+// a normalisation (encode_can_fuse_reference).
+struct RefFusion {
+    const float* rows[kMaxK];
+    int k;
+    const float* alpha;   // device, k floats
+    float* ref_out;       // device, d floats
+};
+bool encode_can_fuse_reference(const CodecGeom& g);
 cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref,
-                          uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp,
+                          const RefFusion* fusion, uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp,
                           FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
 cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref,
                           float* out_a, float* out_b, int sm_count, cudaStream_t st, int* launches);

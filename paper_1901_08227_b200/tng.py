@@ -36,7 +36,7 @@ class Stats(C.Structure):
         ("rounds", C.c_uint64), ("bits_per_coord", C.c_double),
         ("alpha", C.c_double * MAX_HISTORY), ("gram", C.c_double * (MAX_HISTORY * MAX_HISTORY)),
         ("rhs", C.c_double * MAX_HISTORY), ("grad_sq", C.c_double), ("cnz", C.c_double),
-        ("solver_fallback", C.c_uint32), ("reserved", C.c_uint32),
+        ("solver_fallback", C.c_uint32), ("pipeline_error", C.c_uint32),
         ("nonfinite_scales", C.c_uint64), ("kernel_launches", C.c_uint64), ("timed_rounds", C.c_uint64),
         ("ms_dots", C.c_double), ("ms_solve", C.c_double), ("ms_combine", C.c_double),
         ("ms_encode", C.c_double), ("ms_decode", C.c_double),

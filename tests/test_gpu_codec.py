@@ -71,6 +71,19 @@ def test_l2_scale_block128(codec, norm):
     assert_exact(got, want)
 
 
+@pytest.mark.parametrize("codec", CODECS)
+@pytest.mark.parametrize("norm,scale_kind,M", [(tng.NORM_NONE, 0, 1), (tng.NORM_DIFF, 0, 8), (tng.NORM_QUOT, 0, 7),
+                                               (tng.NORM_DIFF, 1, 16), (tng.NORM_QUOT, 1, 3), (tng.NORM_DIFF, 0, 64)])
+def test_long_vectors_take_the_staged_kernel(codec, norm, scale_kind, M):
+    # 17 whole 1024-coordinate chunks go through the bulk-copy pipeline (several fills per
+    # chunk when M > 15, workers split by parity between two warps), then 2 full tiles and
+    # a ragged one through the direct kernel: the wire must not show the seam
+    d = 1024 * 17 + 128 * 2 + 77
+    got, want, st = run_both(d, M, codec, norm, 128, scale_kind=scale_kind, s=5, ld=d + 7 + (4 - (d + 7) % 4) % 4)
+    assert st.pipeline_error == 0
+    assert_exact(got, want)
+
+
 @pytest.mark.parametrize("s", [1, 2, 3, 4, 5, 6, 7])
 def test_qsgd_levels(s):
     got, want, _ = run_both(3001, 4, tng.CODEC_QSGD4, tng.NORM_DIFF, 128, s=s)

@@ -72,10 +72,13 @@ def test_rank_deficient_history_falls_back():
 @pytest.mark.parametrize("mode,K", [(tng.FUSE_LAST, 1), (tng.FUSE_LAST, 3), (tng.FUSE_MEAN, 4)])
 @pytest.mark.parametrize("norm,codec,B", [(tng.NORM_DIFF, tng.CODEC_TERN2, 0), (tng.NORM_QUOT, tng.CODEC_TERN2, 128),
                                           (tng.NORM_DIFF, tng.CODEC_QSGD4, 256), (tng.NORM_DIFF, tng.CODEC_SIGN1, 128)])
-def test_rounds_are_bit_exact_when_the_reference_is(mode, K, norm, codec, B):
+@pytest.mark.parametrize("d", [128 * 9 + 40, 1024 * 18 + 128 * 5 + 40])
+def test_rounds_are_bit_exact_when_the_reference_is(mode, K, norm, codec, B, d):
     # delayed-gradient and window-average references are exact fp32 on both sides,
     # so whole trajectories (codes, scales, aggregates, ring) agree bit for bit
-    d, M, steps = 128 * 9 + 40, 4, 7
+    # (the longer vectors go through the staged kernels, the window average being
+    # combined inside the encode pass)
+    M, steps = 4, 7
     opts = dict(block=B, fuse_mode=mode, seed_lo=21, seed_hi=4, qsgd_levels=4)
     ctx = make_ctx(d, M, K, codec, norm, **opts)
     orc = make_oracle(d, M, K, codec, norm, **opts)
@@ -127,11 +130,12 @@ def test_least_squares_rounds_stage_by_stage(mode, norm, codec, B, K):
 
 
 @pytest.mark.parametrize("mode", [tng.FUSE_LSQ, tng.FUSE_HINDSIGHT])
-def test_step_equals_its_own_stages_and_tracks_the_oracle(mode):
+@pytest.mark.parametrize("d,M,K", [(128 * 64 + 9, 8, 4), (1024 * 40 + 200, 8, 8), (1024 * 21 + 130, 19, 3)])
+def test_step_equals_its_own_stages_and_tracks_the_oracle(mode, d, M, K):
     # tng_step must be exactly fuse -> encode(step = round) -> decode -> push on the GPU,
     # and its aggregates must stay within tolerance of the oracle's trajectory except where a
     # last-bit difference of the reference flips a stochastic rounding (rare).
-    d, M, K, steps = 128 * 64 + 9, 8, 4, 10
+    steps = 10
     opts = dict(block=128, fuse_mode=mode, seed_lo=99)
     a = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_DIFF, **opts)
     b = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_DIFF, **opts)
@@ -155,3 +159,4 @@ def test_step_equals_its_own_stages_and_tracks_the_oracle(mode):
     # a flipped rounding moves one coordinate by R/M (about 1e-3 of the norm here) and stays in the ring
     assert max(rels) < 5e-3
     assert np.median(rels) < TOL
+    assert a.stats().pipeline_error == 0 and b.stats().pipeline_error == 0
