@@ -248,7 +248,7 @@ tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* r
 
 tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, cudaStream_t st) {
     int launches = 0;
-    TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), ref, out_a, out_b, c->sm_count, st, &launches));
+    TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), ref, out_a, out_b, c->fb(), c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
 }

@@ -242,103 +242,113 @@ __global__ void __launch_bounds__(kCodecThreads, 2) encode_kernel(const EncodeAr
 
 // ---------------------------------------------------------------------------
 // Encode fed by the bulk-copy pipeline (one scale per tile, full tiles only).
-// Virtual row list: the rows that make the reference (the k history rows when the
-// reference is combined here, else the reference itself, else nothing), then the M
-// gradient rows.  A chunk of 1024 coordinates = 8 tiles; two warps share a tile and
-// split its workers by parity, so 16 compute warps are busy per CTA.  Both warps of a
-// pair form the reference (the even one stores it).  Everything a warp computes is
-// what encode_tile computes; only where the operands come from differs.
+// Row list: the rows that make the reference (the k history rows when the reference is
+// combined here, else the reference itself, else nothing), then the M gradient rows.
+// A chunk of 2048 coordinates = 16 tiles, one per compute warp; a stage holds up to 8
+// rows of one kind.  Per chunk a warp first forms its tile's reference from the
+// reference fill(s), then encodes the gradient rows fill by fill, eight workers
+// unrolled.  Everything a warp computes is what encode_tile computes; only where the
+// operands come from differs.
 // ---------------------------------------------------------------------------
-constexpr int kEncPipeWarps = 16;
+using EncGeom = PipeGeom<2048, 8, 3>;
+constexpr int kEncPipeWarps = EncGeom::kChunk / kTile;     // 16
 constexpr int kEncPipeThreads = kEncPipeWarps * 32 + 32;   // + the producer warp
+constexpr uint64_t kEncPipeMinChunks = 8;                  // shorter vectors take the direct kernel
 
 struct EncodePipeArgs {
     EncodeArgs e;
     PipeRows rows;
-    int n_pre;          // rows ahead of the gradient rows
 };
 
 template <int CODEC, int NORM, int SCALE, bool FUSEREF>
 __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const EncodePipeArgs pa) {
+    using G = EncGeom;
     extern __shared__ unsigned char dyn_smem[];
     __shared__ float s_alpha[kMaxK];
     const EncodeArgs& a = pa.e;
     if (FUSEREF && threadIdx.x < kMaxK) s_alpha[threadIdx.x] = ((int)threadIdx.x < a.hist_k) ? a.alpha[threadIdx.x] : 0.0f;
-    const PipeSmem pipe = pipe_setup(dyn_smem, kEncPipeWarps);   // ends with __syncthreads
-    const uint64_t nchunks = a.tile_begin / (kChunk / kTile);    // the chunks ahead of the directly read tiles
+    const PipeSmem pipe = pipe_setup<G>(dyn_smem, kEncPipeWarps);   // ends with __syncthreads
+    const uint64_t nchunks = a.tile_begin / kEncPipeWarps;          // the chunks ahead of the directly read tiles
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (warp == kEncPipeWarps) {
         if (lane == 0) {
-            const uint32_t err = pipe_produce(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
+            const uint32_t err = pipe_produce<G>(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
             if (err != kPipeOk) atomicMax(a.pipe_error, err);
         }
         return;
     }
-    const uint32_t tile_in_chunk = (uint32_t)warp >> 1, half = (uint32_t)warp & 1u;
-    const uint32_t my = tile_in_chunk * (kTile * 4u) + (uint32_t)lane * 16u;   // byte offset inside a row chunk
-    const int nrows = pa.rows.nrows, n_pre = pa.n_pre;
+    const uint32_t my = (uint32_t)warp * (kTile * 4u) + (uint32_t)lane * 16u;   // byte offset inside a row chunk
+    const int n_pre = pa.rows.n_pre;
+    const uint32_t M = a.M;
     uint32_t it = 0;
     for (uint64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
-        const uint64_t T = c * (kChunk / kTile) + tile_in_chunk;
-        const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
+        const uint64_t T = c * kEncPipeWarps + (uint32_t)warp;
         const uint64_t q = T * 32u + (uint32_t)lane;
         const uint32_t q_lo = (uint32_t)q, q_hi = (uint32_t)(q >> 32);
-        float4 r = make_float4(0.f, 0.f, 0.f, 0.f), op = r;
-        bool have_op = (NORM == TNG_NORM_NONE);
-        uint32_t rmax = 0;
-        for (int r0 = 0; r0 < nrows; r0 += kStageRows) {
-            const int n = (nrows - r0 < kStageRows) ? nrows - r0 : kStageRows;
-            const uint32_t s = it % kStages, use = it / kStages;
-            if (!__all_sync(kFullMask, mbar_wait(pipe.full[s], use & 1u))) {   // warp-uniform outcome
+        // ---- the reference of the tile
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int p0 = 0; p0 < n_pre; p0 += G::kRows) {
+            const int n = (n_pre - p0 < G::kRows) ? n_pre - p0 : G::kRows;
+            const uint32_t s = it % G::kStages, use = it / G::kStages;
+            if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {   // warp-uniform outcome
                 atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
                 return;
             }
-            const uint32_t base = pipe.data + s * kStageBytes + my;
-            int ri = 0;
-            // rows that make the reference
-            for (; ri < n && r0 + ri < n_pre; ++ri) {
-                const float4 x = lds128(base + (uint32_t)ri * kRowBytes);
-                if (FUSEREF) {
-                    const float al = s_alpha[r0 + ri];
+            const uint32_t base = pipe.data + s * G::kStageBytes + my;
+            if (FUSEREF) {
+                for (int j = 0; j < n; ++j) {
+                    const float4 x = lds128(base + (uint32_t)j * G::kRowBytes);
+                    const float al = s_alpha[p0 + j];
                     r.x = __fmaf_rn(al, x.x, r.x); r.y = __fmaf_rn(al, x.y, r.y);
                     r.z = __fmaf_rn(al, x.z, r.z); r.w = __fmaf_rn(al, x.w, r.w);
-                } else {
-                    r = x;
                 }
-            }
-            if (ri < n && !have_op) {   // the first gradient row is here: the reference is complete
-                if (FUSEREF && half == 0) *reinterpret_cast<float4*>(a.ref_out + i0) = r;
-                if (NORM == TNG_NORM_DIFF) {
-                    op = r;
-                } else {
-                    const float4 den = quot_den4(r, a.quot_eps);
-                    op = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z),
-                                     __fdiv_rn(1.0f, den.w));
-                }
-                have_op = true;
-            }
-            // this warp's workers among the gradient rows of the fill: m = half (mod 2), two at a time
-            int m = r0 + ri - n_pre;                       // worker of stage row ri
-            if (((uint32_t)m & 1u) != half) { ++m; ++ri; }
-            for (; ri + 2 < n; ri += 4, m += 4) {
-                const float4 g0 = lds128(base + (uint32_t)ri * kRowBytes);
-                const float4 g1 = lds128(base + (uint32_t)(ri + 2) * kRowBytes);
-                const uint32_t b0 = encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g0, op, (uint32_t)m, T, q_lo, q_hi, T, lane, 0xFu);
-                const uint32_t b1 = encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g1, op, (uint32_t)m + 2u, T, q_lo, q_hi, T, lane, 0xFu);
-                rmax = max(rmax, max(b0, b1));
-            }
-            if (ri < n) {
-                const float4 g0 = lds128(base + (uint32_t)ri * kRowBytes);
-                rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g0, op, (uint32_t)m, T, q_lo, q_hi, T, lane, 0xFu));
+            } else {
+                r = lds128(base);
             }
             __syncwarp();
-            if (lane == 0) mbar_arrive(pipe.empty[s]);   // this warp has read the stage
+            if (lane == 0) mbar_arrive(pipe.empty(s));
             ++it;
         }
-        // NaN or +inf scales are rare: only then count them, from the scales this warp wrote
+        float4 op = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (NORM != TNG_NORM_NONE) {
+            if (FUSEREF) *reinterpret_cast<float4*>(a.ref_out + (T * kTile + (uint64_t)lane * 4u)) = r;
+            if (NORM == TNG_NORM_DIFF) {
+                op = r;
+            } else {
+                const float4 den = quot_den4(r, a.quot_eps);
+                op = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z),
+                                 __fdiv_rn(1.0f, den.w));
+            }
+        }
+        // ---- the gradient rows, one fill of up to 8 workers at a time
+        uint32_t rmax = 0;
+        for (uint32_t m0 = 0; m0 < M; m0 += G::kRows) {
+            const uint32_t s = it % G::kStages, use = it / G::kStages;
+            if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {
+                atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
+                return;
+            }
+            const uint32_t base = pipe.data + s * G::kStageBytes + my;
+            if (m0 + G::kRows <= M) {
+#pragma unroll
+                for (int k = 0; k < G::kRows; ++k) {
+                    const float4 g = lds128(base + (uint32_t)k * G::kRowBytes);
+                    rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, q_lo, q_hi, T, lane, 0xFu));
+                }
+            } else {
+                for (uint32_t k = 0; m0 + k < M; ++k) {
+                    const float4 g = lds128(base + k * G::kRowBytes);
+                    rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, q_lo, q_hi, T, lane, 0xFu));
+                }
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pipe.empty(s));   // this warp has read the stage
+            ++it;
+        }
+        // NaN or +inf scales are rare: only then count them, from the scales just written
         if (rmax >= 0x7f800000u && lane == 0) {
             unsigned long long bad = 0;
-            for (uint32_t m = half; m < a.M; m += 2) bad += (__float_as_uint(a.scales[(uint64_t)m * a.nblk + T]) >= 0x7f800000u) ? 1ull : 0ull;
+            for (uint32_t m = 0; m < M; ++m) bad += (__float_as_uint(a.scales[(uint64_t)m * a.nblk + T]) >= 0x7f800000u) ? 1ull : 0ull;
             atomicAdd(a.nonfinite, bad);
         }
     }
@@ -394,7 +404,9 @@ struct DecodeArgs {
     const float* ref;
     float* out_a;
     float* out_b;
+    uint32_t* pipe_error;
     uint64_t d, ntile, block;
+    uint64_t tile_begin;   // first tile this launch handles (the staged kernel takes the ones before it)
     uint32_t nblk, wpw;
     uint32_t M;
     uint32_t one;  // 1 as a run-time value: "w << s" is taken as w * (one << s), on the multiplier pipe
@@ -410,21 +422,35 @@ struct DecodeArgs {
 template <int CODEC>
 __device__ __forceinline__ void decode_worker(const uint32_t (&w)[4 * CODEC], const float R, const int levels,
                                               const uint32_t pw, const int lane, float (&acc)[4]) {
-    const bool ok = !scale_is_bad(R);
+    // usable scale: 0 < R < inf, i.e. bit pattern in [1, 0x7f7fffff] (one unsigned compare)
+    const bool ok = (__float_as_uint(R) - 1u) < 0x7f7fffffu;
     const uint32_t Re = ok ? __float_as_uint(R) : 0u;
     const uint32_t okm = ok ? 0x80000000u : 0u;
     if (CODEC == TNG_CODEC_TERN2) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            // sign plane -> sign bit of R; the add is skipped for the zero symbol (acc + 0 == acc)
-            const float sR = __uint_as_float(((w[c * 2 + 1] * pw) & okm) ^ Re);
-            if ((int)(w[c * 2] * pw) < 0) acc[c] = __fadd_rn(acc[c], sR);
+            // sign plane -> sign bit of R; the add is skipped for the zero symbol (acc + 0 == acc).
+            // Written out so that it stays four instructions: a logic op that also sets the
+            // predicate, a multiply (bit -> sign position), a three-input logic op, a predicated add.
+            asm("{\n\t.reg .pred p, pt;\n\t.reg .b32 t, s;\n\t"
+                "setp.eq.u32 pt, 0, 0;\n\t"
+                "lop3.and.b32 t|p, %1, %3, %3, 0xC0, pt;\n\t"   // p = (nonzero word & lane bit) != 0
+                "mul.lo.u32 s, %2, %4;\n\t"                      // lane's sign bit -> bit 31
+                "lop3.b32 s, s, %5, %6, 0x6A;\n\t"              // (s & okm) ^ Re
+                "@p add.rn.f32 %0, %0, s;\n\t}"
+                : "+f"(acc[c])
+                : "r"(w[c * 2]), "r"(w[c * 2 + 1]), "r"(1u << lane), "r"(pw), "r"(okm), "r"(Re));
         }
     } else if (CODEC == TNG_CODEC_SIGN1) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const float sR = __uint_as_float((~(w[c] * pw) & okm) ^ Re);   // plus bit clear -> -R
-            acc[c] = __fadd_rn(acc[c], sR);
+            // plus bit clear -> -R: (~s & okm) ^ Re
+            asm("{\n\t.reg .b32 s;\n\t"
+                "mul.lo.u32 s, %1, %2;\n\t"
+                "lop3.b32 s, s, %3, %4, 0xA6;\n\t"
+                "add.rn.f32 %0, %0, s;\n\t}"
+                : "+f"(acc[c])
+                : "r"(w[c]), "r"(pw), "r"(okm), "r"(Re));
         }
     } else {
         const float step = __fdiv_rn(R, (float)levels);
@@ -439,51 +465,9 @@ __device__ __forceinline__ void decode_worker(const uint32_t (&w)[4 * CODEC], co
     }
 }
 
-template <int CODEC, int N>
-__device__ __forceinline__ void decode_batch(const DecodeArgs& a, const uint32_t* cp, const float* sp, const uint32_t m0,
-                                             const uint32_t pw, const int lane, float (&acc)[4]) {
-    constexpr int kWords = 4 * CODEC;
-    uint4 wv[N][CODEC];
-    float R[N];
-#pragma unroll
-    for (int k = 0; k < N; ++k) {
-        const uint4* wp = reinterpret_cast<const uint4*>(cp + (uint64_t)(m0 + k) * a.wpw);
-#pragma unroll
-        for (int q = 0; q < CODEC; ++q) wv[k][q] = __ldcs(wp + q);
-        R[k] = __ldcs(sp + (uint64_t)(m0 + k) * a.nblk);
-    }
-#pragma unroll
-    for (int k = 0; k < N; ++k) {
-        uint32_t w[kWords];
-#pragma unroll
-        for (int q = 0; q < CODEC; ++q) {
-            w[4 * q + 0] = wv[k][q].x; w[4 * q + 1] = wv[k][q].y; w[4 * q + 2] = wv[k][q].z; w[4 * q + 3] = wv[k][q].w;
-        }
-        decode_worker<CODEC>(w, R[k], a.levels, pw, lane, acc);
-    }
-}
-
-template <int CODEC, int NORM, bool FULL>
-__device__ __forceinline__ void decode_tile(const DecodeArgs& a, const uint64_t T, const int lane) {
-    constexpr int kWords = 4 * CODEC;
-    constexpr int kBatch = (CODEC == TNG_CODEC_QSGD4) ? 2 : 4;   // workers whose code words are in flight together
-    const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
-    const uint32_t pw = a.one << (31 - lane);
-    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
-    if (NORM != TNG_NORM_NONE && a.ref) r = FULL ? *reinterpret_cast<const float4*>(a.ref + i0) : load4(a.ref, i0, a.d);
-    float4 den = make_float4(1.f, 1.f, 1.f, 1.f);
-    if (NORM == TNG_NORM_QUOT) den = quot_den4(r, a.quot_eps);
-    const uint64_t blk = (a.block == (uint64_t)kTile) ? T : (T * kTile) / a.block;
-    // the sum starts from -0 so that (-0) + x == x bit for bit; the ternary path starts from +0
-    // because it skips zero symbols and +0 is what the sum of skipped terms is
-    const float z = (CODEC == TNG_CODEC_TERN2) ? 0.0f : -0.0f;
-    float acc[4] = {z, z, z, z};
-    const uint32_t* cp = a.codes + T * (uint64_t)kWords;
-    const float* sp = a.scales + blk;
-    const uint32_t m_batched = a.M - a.M % kBatch;
-    for (uint32_t m0 = 0; m0 < m_batched; m0 += kBatch) decode_batch<CODEC, kBatch>(a, cp, sp, m0, pw, lane, acc);
-    for (uint32_t m = m_batched; m < a.M; ++m) decode_batch<CODEC, 1>(a, cp, sp, m, pw, lane, acc);
-    // average over the M workers (Algorithm 1), then put the reference back (Eq. 2 / Eq. 3)
+// average over the M workers (Algorithm 1), put the reference back (Eq. 2 / Eq. 3), store
+template <int NORM, bool FULL>
+__device__ __forceinline__ void decode_finish(const DecodeArgs& a, const float (&acc)[4], const float4 r, const uint64_t i0) {
     float4 o;
     if (a.inv_m > 0.0f) {
         o.x = __fmul_rn(acc[0], a.inv_m); o.y = __fmul_rn(acc[1], a.inv_m); o.z = __fmul_rn(acc[2], a.inv_m); o.w = __fmul_rn(acc[3], a.inv_m);
@@ -494,6 +478,7 @@ __device__ __forceinline__ void decode_tile(const DecodeArgs& a, const uint64_t 
     if (NORM == TNG_NORM_DIFF) {
         o.x = __fadd_rn(r.x, o.x); o.y = __fadd_rn(r.y, o.y); o.z = __fadd_rn(r.z, o.z); o.w = __fadd_rn(r.w, o.w);
     } else if (NORM == TNG_NORM_QUOT) {
+        const float4 den = quot_den4(r, a.quot_eps);
         o.x = __fmul_rn(den.x, o.x); o.y = __fmul_rn(den.y, o.y); o.z = __fmul_rn(den.z, o.z); o.w = __fmul_rn(den.w, o.w);
     }
     if (FULL) {
@@ -505,15 +490,132 @@ __device__ __forceinline__ void decode_tile(const DecodeArgs& a, const uint64_t 
     }
 }
 
+// ---------------------------------------------------------------------------
+// Decode kernel.  One warp per tile.  The code words of a tile are the same for all 32
+// lanes, so instead of every lane loading every word, ONE warp-wide load fetches the
+// 16-byte pieces of up to 32/b workers (lane = worker * b + piece), a second one their
+// scales, a third one the lane's four reference values; the words then go through a
+// warp-private shared-memory slot and come back as broadcasts.  The three loads of the
+// warp's next tile are issued before the current tile is decoded, so a warp always has
+// loads in flight while it computes.
+// ---------------------------------------------------------------------------
+constexpr int kDecWarps = kCodecThreads / 32;
+
+struct DecodeSlot {          // per warp
+    uint4 cw[32];
+    float sc[32];
+};
+
+template <int CODEC>
+__device__ __forceinline__ void decode_fetch(const DecodeArgs& a, const uint64_t T, const uint64_t blk, const uint32_t m0,
+                                             const int lane, uint4& cw, float& sc) {
+    constexpr int kRound = 32 / CODEC;            // workers per round
+    const uint32_t m = m0 + (uint32_t)lane / CODEC, piece = (uint32_t)lane % CODEC;
+    cw = make_uint4(0u, 0u, 0u, 0u);
+    sc = 0.0f;
+    if (m < a.M) cw = __ldcs(reinterpret_cast<const uint4*>(a.codes + ((uint64_t)m * a.wpw + T * (uint64_t)(4 * CODEC))) + piece);
+    if (lane < kRound && m0 + (uint32_t)lane < a.M) sc = __ldcs(a.scales + ((uint64_t)(m0 + (uint32_t)lane) * a.nblk + blk));
+}
+
+// decode the `n` workers whose words sit in the slot
+template <int CODEC>
+__device__ __forceinline__ void decode_round(const DecodeSlot* slot, const uint32_t n, const int levels, const uint32_t pw,
+                                             const int lane, float (&acc)[4]) {
+    constexpr int kWords = 4 * CODEC;
+    constexpr int kU = (CODEC == TNG_CODEC_QSGD4) ? 2 : 4;   // workers decoded together
+    uint32_t k = 0;
+    for (; k + kU <= n; k += kU) {
+#pragma unroll
+        for (int kk = 0; kk < kU; ++kk) {
+            uint32_t w[kWords];
+#pragma unroll
+            for (int q = 0; q < CODEC; ++q) {
+                const uint4 t = slot->cw[(k + kk) * CODEC + q];
+                w[4 * q + 0] = t.x; w[4 * q + 1] = t.y; w[4 * q + 2] = t.z; w[4 * q + 3] = t.w;
+            }
+            decode_worker<CODEC>(w, slot->sc[k + kk], levels, pw, lane, acc);
+        }
+    }
+    for (; k < n; ++k) {
+        uint32_t w[kWords];
+#pragma unroll
+        for (int q = 0; q < CODEC; ++q) {
+            const uint4 t = slot->cw[k * CODEC + q];
+            w[4 * q + 0] = t.x; w[4 * q + 1] = t.y; w[4 * q + 2] = t.z; w[4 * q + 3] = t.w;
+        }
+        decode_worker<CODEC>(w, slot->sc[k], levels, pw, lane, acc);
+    }
+}
+
 template <int CODEC, int NORM>
-__global__ void __launch_bounds__(kCodecThreads, 3) decode_kernel(const DecodeArgs a) {
+__global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeArgs a) {
+    __shared__ DecodeSlot slots[kDecWarps];
+    constexpr uint32_t kRound = 32 / CODEC;
     const int lane = threadIdx.x & 31;
-    const uint64_t warps_per_cta = kCodecThreads / 32;
-    const uint64_t nwarps = (uint64_t)gridDim.x * warps_per_cta;
-    const uint64_t gwarp = (uint64_t)blockIdx.x * warps_per_cta + (threadIdx.x >> 5);
+    DecodeSlot* slot = &slots[threadIdx.x >> 5];
+    const uint64_t nwarps = (uint64_t)gridDim.x * kDecWarps;
+    const uint64_t gwarp = (uint64_t)blockIdx.x * kDecWarps + (threadIdx.x >> 5);
     const uint64_t nfull = a.d / kTile;
-    for (uint64_t T = gwarp; T < nfull; T += nwarps) decode_tile<CODEC, NORM, true>(a, T, lane);
-    if (nfull < a.ntile && gwarp == nfull % nwarps) decode_tile<CODEC, NORM, false>(a, nfull, lane);
+    const uint32_t pw = a.one << (31 - lane);
+    const bool tiled = a.block == (uint64_t)kTile;
+    const bool has_ref = (NORM != TNG_NORM_NONE) && a.ref != nullptr;
+    const uint32_t n0 = a.M < kRound ? a.M : kRound;                 // workers of the first round
+    // the sum starts from -0 so that (-0) + x == x bit for bit; the ternary path starts from +0
+    // because it skips zero symbols and +0 is what the sum of skipped terms is
+    const float z = (CODEC == TNG_CODEC_TERN2) ? 0.0f : -0.0f;
+
+    uint64_t T = a.tile_begin + gwarp;
+    uint4 cw = make_uint4(0u, 0u, 0u, 0u);
+    float sc = 0.0f;
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (T < nfull) {
+        decode_fetch<CODEC>(a, T, tiled ? T : (T * kTile) / a.block, 0, lane, cw, sc);
+        if (has_ref) r = *reinterpret_cast<const float4*>(a.ref + (T * kTile + (uint64_t)lane * 4u));
+    }
+    for (; T < nfull; T += nwarps) {
+        slot->cw[lane] = cw;
+        slot->sc[lane] = sc;
+        const float4 rcur = r;
+        __syncwarp();
+        const uint64_t Tn = T + nwarps;
+        if (Tn < nfull) {                                            // next tile's loads go out now
+            decode_fetch<CODEC>(a, Tn, tiled ? Tn : (Tn * kTile) / a.block, 0, lane, cw, sc);
+            if (has_ref) r = *reinterpret_cast<const float4*>(a.ref + (Tn * kTile + (uint64_t)lane * 4u));
+        }
+        float acc[4] = {z, z, z, z};
+        decode_round<CODEC>(slot, n0, a.levels, pw, lane, acc);
+        for (uint32_t m0 = kRound; m0 < a.M; m0 += kRound) {         // more workers than one round holds
+            uint4 cw2;
+            float sc2;
+            decode_fetch<CODEC>(a, T, tiled ? T : (T * kTile) / a.block, m0, lane, cw2, sc2);
+            __syncwarp();
+            slot->cw[lane] = cw2;
+            slot->sc[lane] = sc2;
+            __syncwarp();
+            decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
+        }
+        __syncwarp();                                                // slot is free again
+        decode_finish<NORM, true>(a, acc, rcur, T * kTile + (uint64_t)lane * 4u);
+    }
+    // the ragged last tile
+    if (nfull < a.ntile && gwarp == nfull % nwarps) {
+        const uint64_t Tr = nfull, i0 = Tr * kTile + (uint64_t)lane * 4u;
+        const uint64_t blk = tiled ? Tr : (Tr * kTile) / a.block;
+        float4 rr = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (has_ref) rr = load4(a.ref, i0, a.d);
+        float acc[4] = {z, z, z, z};
+        for (uint32_t m0 = 0; m0 < a.M; m0 += kRound) {
+            uint4 cw2;
+            float sc2;
+            decode_fetch<CODEC>(a, Tr, blk, m0, lane, cw2, sc2);
+            __syncwarp();
+            slot->cw[lane] = cw2;
+            slot->sc[lane] = sc2;
+            __syncwarp();
+            decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
+        }
+        decode_finish<NORM, false>(a, acc, rr, i0);
+    }
 }
 
 // Persistent launch: as many CTAs as fit on the GPU at once (occupancy of this very
@@ -541,36 +643,34 @@ cudaError_t encode_launch_direct(const EncodeArgs& a, int sm_count, cudaStream_t
     return cudaGetLastError();
 }
 
-constexpr uint64_t kEncPipeMinChunks = 16;   // shorter vectors take the direct kernel
-
 // One scale per tile: the whole chunks go through the staged kernel, the remaining tiles
 // (fewer than 8 full ones and a ragged one) through the direct kernel.
 template <int CODEC, int NORM, int SCALE, bool FUSEREF>
 cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t st, int* launches) {
-    const uint64_t nchunks = a0.d / kChunk;
+    const uint64_t nchunks = a0.d / EncGeom::kChunk;
     EncodeArgs a = a0;
     a.tile_begin = 0;
     if (nchunks >= kEncPipeMinChunks) {
         static bool configured = false;   // opt in to the large dynamic shared memory once per instantiation
         auto kern = encode_pipe_kernel<CODEC, NORM, SCALE, FUSEREF>;
         if (!configured) {
-            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
+            cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EncGeom::kSmemBytes);
             if (e != cudaSuccess) return e;
             configured = true;
         }
         EncodePipeArgs pa;
         pa.e = a;
-        pa.e.tile_begin = nchunks * (kChunk / kTile);
+        pa.e.tile_begin = nchunks * kEncPipeWarps;
         pa.rows.nrows = 0;
         if (FUSEREF) {
             for (int j = 0; j < a.hist_k; ++j) pa.rows.row[pa.rows.nrows++] = a.hist[j];
         } else if (NORM != TNG_NORM_NONE && a.ref) {
             pa.rows.row[pa.rows.nrows++] = a.ref;
         }
-        pa.n_pre = pa.rows.nrows;
+        pa.rows.n_pre = pa.rows.nrows;
         for (uint32_t m = 0; m < a.M; ++m) pa.rows.row[pa.rows.nrows++] = a.grads + (uint64_t)m * a.ld;
         const int grid = (int)(nchunks < (uint64_t)sm_count ? nchunks : (uint64_t)sm_count);
-        kern<<<grid, kEncPipeThreads, kPipeSmemBytes, st>>>(pa);
+        kern<<<grid, kEncPipeThreads, EncGeom::kSmemBytes, st>>>(pa);
         ++*launches;
         cudaError_t e = cudaGetLastError();
         if (e != cudaSuccess) return e;
@@ -620,21 +720,22 @@ cudaError_t encode_dispatch(const EncodeArgs& a, int codec, int norm, int scale,
 }
 
 template <int CODEC, int NORM>
-cudaError_t decode_launch(const DecodeArgs& a, int sm_count, cudaStream_t st) {
+cudaError_t decode_launch(const DecodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
     static int per_tiles_grid = 0;
     auto kern = decode_kernel<CODEC, NORM>;
     if (per_tiles_grid == 0) per_tiles_grid = persistent_grid(kern, ~0ull >> 8, sm_count);
-    const uint64_t want = (a.ntile + 7) / 8;
+    const uint64_t want = (a.ntile - a.tile_begin + 7) / 8;
     const int grid = (int)(want < (uint64_t)per_tiles_grid ? (want ? want : 1) : (uint64_t)per_tiles_grid);
     kern<<<grid, kCodecThreads, 0, st>>>(a);
+    ++*launches;
     return cudaGetLastError();
 }
 template <int CODEC>
-cudaError_t decode_dispatch_norm(const DecodeArgs& a, int norm, int sm_count, cudaStream_t st) {
+cudaError_t decode_dispatch_norm(const DecodeArgs& a, int norm, int sm_count, cudaStream_t st, int* launches) {
     switch (norm) {
-        case TNG_NORM_DIFF: return decode_launch<CODEC, TNG_NORM_DIFF>(a, sm_count, st);
-        case TNG_NORM_QUOT: return decode_launch<CODEC, TNG_NORM_QUOT>(a, sm_count, st);
-        default: return decode_launch<CODEC, TNG_NORM_NONE>(a, sm_count, st);
+        case TNG_NORM_DIFF: return decode_launch<CODEC, TNG_NORM_DIFF>(a, sm_count, st, launches);
+        case TNG_NORM_QUOT: return decode_launch<CODEC, TNG_NORM_QUOT>(a, sm_count, st, launches);
+        default: return decode_launch<CODEC, TNG_NORM_NONE>(a, sm_count, st, launches);
     }
 }
 
@@ -697,19 +798,19 @@ cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, c
 }
 
 cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref,
-                          float* out_a, float* out_b, int sm_count, cudaStream_t st, int* launches) {
+                          float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
     DecodeArgs a;
     a.codes = codes; a.scales = scales; a.ref = ref; a.out_a = out_a; a.out_b = out_b;
+    a.pipe_error = &fb->pipe_error; a.tile_begin = 0;
     a.d = g.d; a.ntile = g.ntile; a.nblk = (uint32_t)g.nblk; a.block = g.block; a.wpw = (uint32_t)g.wpw; a.M = g.M;
     a.one = 1u; a.levels = g.levels; a.quot_eps = g.quot_eps;
     a.inv_m = ((g.M & (g.M - 1)) == 0) ? 1.0f / (float)g.M : 0.0f;
     cudaError_t e;
     switch (g.codec) {
-        case TNG_CODEC_SIGN1: e = decode_dispatch_norm<TNG_CODEC_SIGN1>(a, g.norm, sm_count, st); break;
-        case TNG_CODEC_TERN2: e = decode_dispatch_norm<TNG_CODEC_TERN2>(a, g.norm, sm_count, st); break;
-        default: e = decode_dispatch_norm<TNG_CODEC_QSGD4>(a, g.norm, sm_count, st); break;
+        case TNG_CODEC_SIGN1: e = decode_dispatch_norm<TNG_CODEC_SIGN1>(a, g.norm, sm_count, st, launches); break;
+        case TNG_CODEC_TERN2: e = decode_dispatch_norm<TNG_CODEC_TERN2>(a, g.norm, sm_count, st, launches); break;
+        default: e = decode_dispatch_norm<TNG_CODEC_QSGD4>(a, g.norm, sm_count, st, launches); break;
     }
-    ++*launches;
     return e;
 }
 

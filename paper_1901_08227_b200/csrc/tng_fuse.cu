@@ -89,7 +89,8 @@ __device__ __forceinline__ void dots_finish(const double (&acc)[kAcc], const Dot
 // of the vectors (d mod 1024) is read directly.
 // ---------------------------------------------------------------------------
 constexpr int kDotsPipeThreads = kDotsThreads + 32;   // 8 consumer warps + 1 producer warp
-constexpr uint64_t kDotsPipeMinCoords = 16 * kChunk;    // shorter vectors take the direct kernel
+using DotsGeom = PipeGeom<1024, 16, 3>;                // 64 KiB stages: a chunk of 1024 coordinates of 16 rows
+constexpr uint64_t kDotsPipeMinCoords = 16 * DotsGeom::kChunk;   // shorter vectors take the direct kernel
 
 struct DotsPipeArgs {
     DotsArgs base;      // rows_a = history rows, grads/ld/M, partials, fb, dst
@@ -132,9 +133,10 @@ __global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const Do
     constexpr int kPairs = NA * (NA + 1) / 2;
     constexpr int kAcc = kPairs + NA + 1;
     const DotsArgs& a = pa.base;
-    const PipeSmem pipe = pipe_setup(dyn_smem, kDotsThreads / 32);
+    using G = DotsGeom;
+    const PipeSmem pipe = pipe_setup<G>(dyn_smem, kDotsThreads / 32);
     const bool with_g = a.grads != nullptr;
-    const uint64_t nchunks = a.d / kChunk;
+    const uint64_t nchunks = a.d / G::kChunk;
     const int tid = threadIdx.x;
     double acc[kAcc];
 #pragma unroll
@@ -143,44 +145,43 @@ __global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const Do
     if (tid >= kDotsThreads) {
         // ---- producer warp: one thread feeds the stages
         if (tid == kDotsThreads) {
-            const uint32_t err = pipe_produce(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
+            const uint32_t err = pipe_produce<G>(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
             if (err != kPipeOk) atomicMax(&a.fb->pipe_error, err);
         }
     } else {
-        // ---- consumers
+        // ---- consumers: fill 0 of a chunk holds the NA history rows, the others gradient rows
         const int lane = tid & 31;
         const uint32_t my = (uint32_t)tid * 16u;                  // byte offset of the thread's float4 inside a row chunk
-        const int nrows = pa.rows.nrows;
+        const int ngrad = pa.rows.nrows - pa.rows.n_pre;
         uint32_t it = 0;
         bool alive = true;
         for (uint64_t c = blockIdx.x; c < nchunks && alive; c += gridDim.x) {
             float4 ha[NA];
             float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), gq = make_float4(0.f, 0.f, 0.f, 0.f);
-            for (int r0 = 0; r0 < nrows; r0 += kStageRows) {
-                const int n = (nrows - r0 < kStageRows) ? nrows - r0 : kStageRows;
-                const uint32_t s = it % kStages, use = it / kStages;
-                if (!__all_sync(kFullMask, mbar_wait(pipe.full[s], use & 1u))) {   // warp-uniform outcome
+            for (int g0 = -G::kRows; g0 < ngrad; g0 += G::kRows) {   // g0 < 0: the history fill
+                const uint32_t s = it % G::kStages, use = it / G::kStages;
+                if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {   // warp-uniform outcome
                     atomicMax(&a.fb->pipe_error, (uint32_t)kPipeFullTimeout);
                     alive = false;
                     break;
                 }
-                const uint32_t base = pipe.data + s * kStageBytes + my;
-                int r = 0;
-                if (r0 == 0) {
+                const uint32_t base = pipe.data + s * G::kStageBytes + my;
+                if (g0 < 0) {
 #pragma unroll
-                    for (int j = 0; j < NA; ++j) ha[j] = lds128(base + (uint32_t)j * kRowBytes);
-                    r = NA;
+                    for (int j = 0; j < NA; ++j) ha[j] = lds128(base + (uint32_t)j * G::kRowBytes);
+                } else {
+                    const int n = (ngrad - g0 < G::kRows) ? ngrad - g0 : G::kRows;
+                    for (int r = 0; r < n; ++r) grad_sums(gs, gq, lds128(base + (uint32_t)r * G::kRowBytes));
                 }
-                for (; r < n; ++r) grad_sums(gs, gq, lds128(base + (uint32_t)r * kRowBytes));
                 __syncwarp();
-                if (lane == 0) mbar_arrive(pipe.empty[s]);       // this warp has read the stage
+                if (lane == 0) mbar_arrive(pipe.empty(s));       // this warp has read the stage
                 ++it;
             }
             if (alive) dots_accum4<NA>(ha, gs, gq, with_g, acc);
         }
         // ---- ragged end: coordinates [nchunks*1024, d) straight from global memory
         const uint64_t ngroups = (a.d + 3) / 4;
-        for (uint64_t grp = nchunks * (kChunk / 4) + (uint64_t)blockIdx.x * kDotsThreads + tid; grp < ngroups;
+        for (uint64_t grp = nchunks * (G::kChunk / 4) + (uint64_t)blockIdx.x * kDotsThreads + tid; grp < ngroups;
              grp += (uint64_t)gridDim.x * kDotsThreads) {
             const uint64_t i0 = grp * 4;
             float4 ha[NA];
@@ -280,11 +281,11 @@ template <int NA>
 cudaError_t dots_pipe(const DotsPipeArgs& pa, int grid, cudaStream_t st) {
     static bool configured = false;   // opt in to the large dynamic shared memory once per instantiation
     if (!configured) {
-        cudaError_t e = cudaFuncSetAttribute(dots_pipe_kernel<NA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kPipeSmemBytes);
+        cudaError_t e = cudaFuncSetAttribute(dots_pipe_kernel<NA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DotsGeom::kSmemBytes);
         if (e != cudaSuccess) return e;
         configured = true;
     }
-    dots_pipe_kernel<NA><<<grid, kDotsPipeThreads, kPipeSmemBytes, st>>>(pa);
+    dots_pipe_kernel<NA><<<grid, kDotsPipeThreads, DotsGeom::kSmemBytes, st>>>(pa);
     return cudaGetLastError();
 }
 cudaError_t dots_pipe_n(int n, const DotsPipeArgs& pa, int grid, cudaStream_t st) {
@@ -491,9 +492,10 @@ cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float
         pa.base = a;
         pa.rows.nrows = 0;
         for (int j = 0; j < k; ++j) pa.rows.row[pa.rows.nrows++] = rows[j];
+        pa.rows.n_pre = k;
         if (grads)
             for (uint32_t m = 0; m < M; ++m) pa.rows.row[pa.rows.nrows++] = grads + (uint64_t)m * ld;
-        const uint64_t nchunks = d / kChunk;
+        const uint64_t nchunks = d / DotsGeom::kChunk;
         const int pgrid = (int)(nchunks < (uint64_t)sm_count ? nchunks : (uint64_t)sm_count);
         e = dots_pipe_n(k, pa, pgrid, st);
         ++*launches;

@@ -71,6 +71,6 @@ cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, c
                           const RefFusion* fusion, uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp,
                           FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
 cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref,
-                          float* out_a, float* out_b, int sm_count, cudaStream_t st, int* launches);
+                          float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
 
 }  // namespace tng

@@ -20,12 +20,17 @@
 
 namespace tng {
 
-constexpr int kChunk = 1024;                 // coordinates per row per stage (4 KiB)
-constexpr int kStageRows = 16;               // rows per stage (64 KiB)
-constexpr int kStages = 3;                   // stages per CTA (192 KiB)
-constexpr uint32_t kRowBytes = kChunk * 4u;
-constexpr uint32_t kStageBytes = kStageRows * kRowBytes;
-constexpr uint32_t kPipeSmemBytes = kStages * kStageBytes + 1024;   // + barriers, alignment slack
+// Geometry of one pipeline: CHUNK coordinates of ROWS rows per stage, STAGES stages.
+template <int CHUNK, int ROWS, int STAGES>
+struct PipeGeom {
+    static constexpr int kChunk = CHUNK;
+    static constexpr int kRows = ROWS;
+    static constexpr int kStages = STAGES;
+    static constexpr uint32_t kRowBytes = CHUNK * 4u;
+    static constexpr uint32_t kStageBytes = ROWS * kRowBytes;
+    static constexpr uint32_t kSmemBytes = STAGES * kStageBytes + 1024;   // + barriers, alignment slack
+};
+constexpr int kMaxStages = 4;
 constexpr int kSpinLimit = 1 << 22;          // polls of try_wait (each may itself block briefly)
 
 enum PipeError : uint32_t { kPipeOk = 0, kPipeFullTimeout = 1, kPipeEmptyTimeout = 2 };
@@ -78,30 +83,26 @@ __device__ __forceinline__ float4 lds128(uint32_t addr) {
     return v;
 }
 
-// Shared-memory footprint of one pipeline: stage data (1 KiB aligned) then the barriers.
+// Shared-memory footprint of one pipeline: stage data (128-byte aligned) then the barriers.
 struct PipeSmem {
     uint32_t data;                 // shared address of stage 0
-    uint32_t full[kStages];
-    uint32_t empty[kStages];
+    uint32_t bars;                 // full[s] at bars + 16 s, empty[s] at bars + 16 s + 8
+    __device__ __forceinline__ uint32_t full(uint32_t s) const { return bars + 16u * s; }
+    __device__ __forceinline__ uint32_t empty(uint32_t s) const { return bars + 16u * s + 8u; }
 };
 
 // Carve the dynamic shared memory and initialise the barriers (thread 0), then sync.
 // `consumer_arrivals` = arrivals that free a stage (one per consumer warp).
+template <class G>
 __device__ __forceinline__ PipeSmem pipe_setup(unsigned char* dyn_smem, uint32_t consumer_arrivals) {
     PipeSmem p;
-    const uint32_t base = (smem_u32(dyn_smem) + 127u) & ~127u;
-    p.data = base;
-    const uint32_t bars = base + kStages * kStageBytes;
-#pragma unroll
-    for (int s = 0; s < kStages; ++s) {
-        p.full[s] = bars + 16u * s;
-        p.empty[s] = bars + 16u * s + 8u;
-    }
+    p.data = (smem_u32(dyn_smem) + 127u) & ~127u;
+    p.bars = p.data + G::kStages * G::kStageBytes;
     if (threadIdx.x == 0) {
 #pragma unroll
-        for (int s = 0; s < kStages; ++s) {
-            mbar_init(p.full[s], 1);
-            mbar_init(p.empty[s], consumer_arrivals);
+        for (int s = 0; s < G::kStages; ++s) {
+            mbar_init(p.full(s), 1);
+            mbar_init(p.empty(s), consumer_arrivals);
         }
         mbar_init_fence();
     }
@@ -109,29 +110,65 @@ __device__ __forceinline__ PipeSmem pipe_setup(unsigned char* dyn_smem, uint32_t
     return p;
 }
 
-// Row source list of one launch: pointer of each virtual row (all 16-byte aligned).
-// A "fill" is up to kStageRows consecutive rows of the list for one chunk of coordinates.
+// Same with the stage count and size chosen at launch time (stage_bytes a multiple of 128).
+__device__ __forceinline__ PipeSmem pipe_setup_rt(unsigned char* dyn_smem, uint32_t nstages, uint32_t stage_bytes,
+                                                  uint32_t consumer_arrivals) {
+    PipeSmem p;
+    p.data = (smem_u32(dyn_smem) + 127u) & ~127u;
+    p.bars = p.data + nstages * stage_bytes;
+    if (threadIdx.x == 0) {
+        for (uint32_t s = 0; s < nstages; ++s) {
+            mbar_init(p.full(s), 1);
+            mbar_init(p.empty(s), consumer_arrivals);
+        }
+        mbar_init_fence();
+    }
+    __syncthreads();
+    return p;
+}
+
+__device__ __forceinline__ uint4 lds128u(uint32_t addr) {
+    uint4 v;
+    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
+    return v;
+}
+__device__ __forceinline__ float lds32(uint32_t addr) {
+    float v;
+    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
+    return v;
+}
+
+// Row source list of one launch: pointer of each row (all 16-byte aligned): first n_pre
+// rows of one kind (history / reference), then the gradient rows.  A "fill" is up to ROWS
+// consecutive rows of ONE kind for one chunk of coordinates: fills never mix the two kinds,
+// so a chunk takes ceil(n_pre / ROWS) + ceil((nrows - n_pre) / ROWS) fills, in that order.
 struct PipeRows {
     const float* row[80];          // up to 16 history rows + 64 gradient rows
     int nrows;
+    int n_pre;
 };
 
 // Producer side, run by ONE thread: for chunk indices c = first, first + stride, ... < nchunks
 // and for each fill of the row list, wait for a free stage and issue the row copies.
 // Returns kPipeOk or the error that stopped it.
+template <class G>
 __device__ __forceinline__ uint32_t pipe_produce(const PipeSmem& p, const PipeRows& rows, uint64_t first, uint64_t stride,
                                                  uint64_t nchunks) {
     uint32_t it = 0;
     for (uint64_t c = first; c < nchunks; c += stride) {
-        for (int r0 = 0; r0 < rows.nrows; r0 += kStageRows) {
-            const int n = (rows.nrows - r0 < kStageRows) ? rows.nrows - r0 : kStageRows;
-            const uint32_t s = it % kStages, use = it / kStages;
+        int r0 = 0;
+        while (r0 < rows.nrows) {
+            const int seg_end = (r0 < rows.n_pre) ? rows.n_pre : rows.nrows;
+            const int n = (seg_end - r0 < G::kRows) ? seg_end - r0 : G::kRows;
+            const uint32_t s = it % G::kStages, use = it / G::kStages;
             // a stage is free once its previous use has been consumed (parity of use - 1)
-            if (use > 0 && !mbar_wait(p.empty[s], (use - 1) & 1u)) return kPipeEmptyTimeout;
-            mbar_expect_tx(p.full[s], (uint32_t)n * kRowBytes);
-            const uint32_t dst = p.data + s * kStageBytes;
-            for (int r = 0; r < n; ++r) bulk_load(dst + (uint32_t)r * kRowBytes, rows.row[r0 + r] + c * kChunk, kRowBytes, p.full[s]);
+            if (use > 0 && !mbar_wait(p.empty(s), (use - 1) & 1u)) return kPipeEmptyTimeout;
+            mbar_expect_tx(p.full(s), (uint32_t)n * G::kRowBytes);
+            const uint32_t dst = p.data + s * G::kStageBytes;
+            for (int r = 0; r < n; ++r)
+                bulk_load(dst + (uint32_t)r * G::kRowBytes, rows.row[r0 + r] + c * G::kChunk, G::kRowBytes, p.full(s));
             ++it;
+            r0 += n;
         }
     }
     return kPipeOk;

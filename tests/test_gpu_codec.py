@@ -74,11 +74,13 @@ def test_l2_scale_block128(codec, norm):
 @pytest.mark.parametrize("codec", CODECS)
 @pytest.mark.parametrize("norm,scale_kind,M", [(tng.NORM_NONE, 0, 1), (tng.NORM_DIFF, 0, 8), (tng.NORM_QUOT, 0, 7),
                                                (tng.NORM_DIFF, 1, 16), (tng.NORM_QUOT, 1, 3), (tng.NORM_DIFF, 0, 64)])
-def test_long_vectors_take_the_staged_kernel(codec, norm, scale_kind, M):
-    # 17 whole 1024-coordinate chunks go through the bulk-copy pipeline (several fills per
-    # chunk when M > 15, workers split by parity between two warps), then 2 full tiles and
-    # a ragged one through the direct kernel: the wire must not show the seam
-    d = 1024 * 17 + 128 * 2 + 77
+@pytest.mark.parametrize("d", [1024 * 17 + 128 * 2 + 77, 2048 * 9 + 128 * 3 + 50])
+def test_long_vectors_take_the_staged_kernels(codec, norm, scale_kind, M, d):
+    # whole 2048-coordinate chunks go through the bulk-copy pipelines (several fills per
+    # chunk when M > 8), the remaining full tiles and the ragged one through the direct
+    # kernels: neither the wire nor the aggregate may show the seam.  The second length has
+    # a tile count that is a multiple of 4, which the staged decode needs; the first one
+    # decodes with the direct kernel.
     got, want, st = run_both(d, M, codec, norm, 128, scale_kind=scale_kind, s=5, ld=d + 7 + (4 - (d + 7) % 4) % 4)
     assert st.pipeline_error == 0
     assert_exact(got, want)
