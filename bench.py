@@ -39,16 +39,33 @@ WORKLOADS = {
 }
 
 
-def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True):
-    """Bytes per coordinate each kernel of one round has to move (reads + writes)."""
+def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True, ref_in_encode=True):
+    """Bytes per coordinate each kernel of one round has to move (reads + writes).
+
+    dots    reads the K ring rows and the M gradient rows;
+    encode  reads the M gradient rows and writes the wire (codes + scales); with the reference
+            combine folded into it (block 128) it also reads the K ring rows and writes the
+            reference, otherwise it reads the reference a separate combine pass wrote;
+    decode  reads the wire and the reference, writes the new ring entry (and the caller's copy)."""
     wire = M * bits / 8.0 + 4.0 * M / block
     per = {}
     if fuse == "lsq":
         per["dots"] = 4.0 * K + 4.0 * M
-        per["combine"] = 4.0 * K + 4.0
-    per["encode"] = 4.0 * M + 4.0 + wire
+        if ref_in_encode:
+            per["encode"] = 4.0 * K + 4.0 * M + 4.0 + wire
+        else:
+            per["combine"] = 4.0 * K + 4.0
+            per["encode"] = 4.0 * M + 4.0 + wire
+    else:
+        per["encode"] = 4.0 * M + 4.0 + wire
     per["decode"] = wire + 4.0 + 4.0 + (4.0 if user_out else 0.0)
     return per
+
+
+# dram__bytes_read.sum + dram__bytes_write.sum per coordinate of the dominant kernel, from the ncu
+# capture summarised under profiles/ (taken at d = 2^24 and scaled by d: every kernel streams each
+# coordinate once).  None = the kernel changed after the capture.
+NCU_TRAFFIC_BYTES_PER_COORD = {"encode": None, "dots": None, "decode": None}
 
 
 def measured_hbm_peak():
@@ -261,7 +278,8 @@ def run_ours(args, name, cfg):
     n0, n1 = st0.timed_rounds, st1.timed_rounds
     def stage_ms(field):
         return (getattr(st1, field) * n1 - getattr(st0, field) * n0) / max(n1 - n0, 1)
-    per_coord = algorithmic_bytes_per_coord(M, K, bits, cfg["block"], cfg["fuse"])
+    ref_in_encode = cfg["block"] == 128 and cfg["norm"] != "none" and stage_ms("ms_combine") == 0.0
+    per_coord = algorithmic_bytes_per_coord(M, K, bits, cfg["block"], cfg["fuse"], ref_in_encode=ref_in_encode)
     peak, peak_src = measured_hbm_peak()
     kernels = {}
     for kname, field in (("dots", "ms_dots"), ("combine", "ms_combine"), ("encode", "ms_encode"), ("decode", "ms_decode")):
@@ -270,9 +288,12 @@ def run_ours(args, name, cfg):
         ms = stage_ms(field)
         gbs = per_coord[kname] * d / (ms * 1e-3) / 1e9 if ms > 0 else None
         kernels[kname] = {"ms": ms, "bytes_per_coord": per_coord[kname], "GBps": gbs, "frac_of_measured": gbs / peak if gbs else None}
+    if ref_in_encode and "encode" in kernels:
+        kernels["encode"]["includes"] = "reference combine (ring rows -> reference) folded into the encode pass"
     kernels["solve"] = {"ms": stage_ms("ms_solve")}
     dominant = max((k for k in kernels if "bytes_per_coord" in kernels[k]), key=lambda k: kernels[k]["ms"])
-    traffic = {"dots": None, "combine": None, "encode": None, "decode": None}.get(dominant)
+    tpc = NCU_TRAFFIC_BYTES_PER_COORD.get(dominant)
+    traffic = tpc * d if tpc is not None else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["GBps"], "peak": peak, "unit": "GB/s",
                 "frac": kernels[dominant]["frac_of_measured"], "peak_source": peak_src, "traffic": traffic,
                 "algorithmic_bytes_per_launch": per_coord[dominant] * d}

@@ -62,13 +62,9 @@ __device__ __forceinline__ float absmax_nan2(float a, float b) {
 // The integer/logic pipe is the busy one in this kernel (Philox xors, compares,
 // ballots), so work that can run on the multiplier pipe is put there: addresses are
 // 32 x 32 -> 64 multiply-adds and the uniform's shift is a high multiply.
-template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL>
-__device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const float4 g, const float4 op,
-                                                  const uint32_t m, const uint64_t T, const uint32_t q_lo,
-                                                  const uint32_t q_hi, const uint64_t blk, const int lane,
-                                                  const uint32_t valid) {
-    // ---- normalise: v = g - r (Eq. 2), v = g * (1/den) (Eq. 3), or v = g
-    float v[4];
+// v = g - r (Eq. 2), v = g * (1/den) (Eq. 3), or v = g
+template <int NORM>
+__device__ __forceinline__ void encode_normalise(const float4 g, const float4 op, float (&v)[4]) {
     if (NORM == TNG_NORM_DIFF) {
         v[0] = __fsub_rn(g.x, op.x); v[1] = __fsub_rn(g.y, op.y); v[2] = __fsub_rn(g.z, op.z); v[3] = __fsub_rn(g.w, op.w);
     } else if (NORM == TNG_NORM_QUOT) {
@@ -76,31 +72,25 @@ __device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const flo
     } else {
         v[0] = g.x; v[1] = g.y; v[2] = g.z; v[3] = g.w;
     }
-    // ---- scale of the block
-    float R;
-    if (PHASE != kPhaseQuant) {
-        float stat;
-        if (SCALE == 0) {
-            const float mx = absmax_nan2(absmax_nan2(v[0], v[1]), absmax_nan2(v[2], v[3]));
-            // non-negative floats and NaNs order like their bit patterns
-            stat = __uint_as_float(__reduce_max_sync(kFullMask, __float_as_uint(mx)));
-        } else {
-            stat = warp_sumsq_tree(v[0], v[1], v[2], v[3]);
-        }
-        if (PHASE == kPhaseStat) {
-            if (lane == 0) a.tile_stat[(uint64_t)m * a.ntile + T] = stat;
-            return 0u;
-        }
-        R = (SCALE == 0) ? stat : __fsqrt_rn(stat);
-    } else {
-        R = __ldg(a.scales + (uint64_t)m * a.nblk + blk);
-    }
+}
 
-    // ---- stochastic rounding: one Philox call per lane, word c for coordinate 4j+c
-    const uint4 x = philox4x32_10_rk(q_lo, q_hi, m, a.step, a.rk);
+// the tile's statistic: max |v| (NaN wins) or the pairwise-tree sum of squares
+template <int SCALE>
+__device__ __forceinline__ float encode_tile_stat(const float (&v)[4]) {
+    if (SCALE == 0) {
+        const float mx = absmax_nan2(absmax_nan2(v[0], v[1]), absmax_nan2(v[2], v[3]));
+        // non-negative floats and NaNs order like their bit patterns
+        return __uint_as_float(__reduce_max_sync(kFullMask, __float_as_uint(mx)));
+    }
+    return warp_sumsq_tree(v[0], v[1], v[2], v[3]);
+}
+
+// Stochastic rounding of the lane's four values with scale R; x = the lane's Philox call,
+// word c for coordinate 4j+c.  The ballots leave every code word of the tile in every lane.
+template <int CODEC, bool FULL>
+__device__ __forceinline__ void encode_quantise(const EncodeArgs& a, const float (&v)[4], const float R, const uint4 x,
+                                                const uint32_t valid, uint32_t (&w)[4 * CODEC]) {
     const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
-    constexpr int kWords = 4 * CODEC;
-    uint32_t w[kWords];
 #pragma unroll
     for (int c = 0; c < 4; ++c) {
         // u = (x >> 8) * 2^-24
@@ -131,7 +121,41 @@ __device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const flo
             w[c * 4 + 3] = __ballot_sync(kFullMask, neg);
         }
     }
-    // every lane holds all words of the tile; lane 0 writes them (and the scale)
+}
+
+template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL>
+__device__ __forceinline__ bool encode_symbols(const EncodeArgs& a, const float4 g, const float4 op,
+                                               const uint32_t m, const uint64_t T, const uint4 x, const uint64_t blk,
+                                               const int lane, const uint32_t valid, uint32_t (&w)[4 * CODEC], float& R) {
+    float v[4];
+    encode_normalise<NORM>(g, op, v);
+    if (PHASE != kPhaseQuant) {
+        const float stat = encode_tile_stat<SCALE>(v);
+        if (PHASE == kPhaseStat) {
+            if (lane == 0) a.tile_stat[(uint64_t)m * a.ntile + T] = stat;
+            R = 0.0f;
+            return false;
+        }
+        R = (SCALE == 0) ? stat : __fsqrt_rn(stat);
+    } else {
+        R = __ldg(a.scales + (uint64_t)m * a.nblk + blk);
+    }
+    encode_quantise<CODEC, FULL>(a, v, R, x, valid, w);
+    return true;
+}
+
+// encode_symbols, then lane 0 writes the words every lane holds (and the scale)
+template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL>
+__device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const float4 g, const float4 op,
+                                                  const uint32_t m, const uint64_t T, const uint32_t q_lo,
+                                                  const uint32_t q_hi, const uint64_t blk, const int lane,
+                                                  const uint32_t valid) {
+    constexpr int kWords = 4 * CODEC;
+    uint32_t w[kWords];
+    float R;
+    uint4 x = make_uint4(0u, 0u, 0u, 0u);
+    if (PHASE != kPhaseStat) x = philox4x32_10_rk(q_lo, q_hi, m, a.step, a.rk);
+    if (!encode_symbols<CODEC, NORM, SCALE, PHASE, FULL>(a, g, op, m, T, x, blk, lane, valid, w, R)) return 0u;
     if (lane == 0) {
         uint4* dst = reinterpret_cast<uint4*>(a.codes + ((uint64_t)m * a.wpw + T * (uint64_t)kWords));
 #pragma unroll
@@ -240,6 +264,15 @@ __global__ void __launch_bounds__(kCodecThreads, 2) encode_kernel(const EncodeAr
     if (nfull < a.ntile && gwarp == nfull % nwarps) encode_tile<CODEC, NORM, SCALE, PHASE, false, FUSEREF>(a, s_alpha, nfull, lane);
 }
 
+// Predicated 16-byte stores of a tile's code words (no branch around them).
+template <int CODEC>
+__device__ __forceinline__ void store_words_if(const bool pred, uint32_t* dst, const uint32_t (&w)[4 * CODEC]) {
+#pragma unroll
+    for (int q4 = 0; q4 < CODEC; ++q4)
+        asm volatile("{\n\t.reg .pred p;\n\tsetp.ne.u32 p, %0, 0;\n\t@p st.global.cs.v4.u32 [%1], {%2, %3, %4, %5};\n\t}" ::"r"((uint32_t)pred),
+                     "l"(dst + 4 * q4), "r"(w[4 * q4]), "r"(w[4 * q4 + 1]), "r"(w[4 * q4 + 2]), "r"(w[4 * q4 + 3]));
+}
+
 // ---------------------------------------------------------------------------
 // Encode fed by the bulk-copy pipeline (one scale per tile, full tiles only).
 // Row list: the rows that make the reference (the k history rows when the reference is
@@ -254,6 +287,7 @@ using EncGeom = PipeGeom<2048, 8, 3>;
 constexpr int kEncPipeWarps = EncGeom::kChunk / kTile;     // 16
 constexpr int kEncPipeThreads = kEncPipeWarps * 32 + 32;   // + the producer warp
 constexpr uint64_t kEncPipeMinChunks = 8;                  // shorter vectors take the direct kernel
+constexpr int kPhiloxBatch = 2;                            // Philox calls whose rounds are interleaved
 
 struct EncodePipeArgs {
     EncodeArgs e;
@@ -278,6 +312,9 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
         return;
     }
     const uint32_t my = (uint32_t)warp * (kTile * 4u) + (uint32_t)lane * 16u;   // byte offset inside a row chunk
+    // the stages as ordinary shared memory: plain loads, which the compiler may interleave freely
+    // with the arithmetic of neighbouring workers (the barrier waits are memory fences for it)
+    const unsigned char* stages = dyn_smem + (pipe.data - smem_u32(dyn_smem));
     const int n_pre = pa.rows.n_pre;
     const uint32_t M = a.M;
     uint32_t it = 0;
@@ -294,16 +331,16 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                 atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
                 return;
             }
-            const uint32_t base = pipe.data + s * G::kStageBytes + my;
+            const unsigned char* base = stages + s * G::kStageBytes + my;
             if (FUSEREF) {
                 for (int j = 0; j < n; ++j) {
-                    const float4 x = lds128(base + (uint32_t)j * G::kRowBytes);
+                    const float4 x = *reinterpret_cast<const float4*>(base + (uint32_t)j * G::kRowBytes);
                     const float al = s_alpha[p0 + j];
                     r.x = __fmaf_rn(al, x.x, r.x); r.y = __fmaf_rn(al, x.y, r.y);
                     r.z = __fmaf_rn(al, x.z, r.z); r.w = __fmaf_rn(al, x.w, r.w);
                 }
             } else {
-                r = lds128(base);
+                r = *reinterpret_cast<const float4*>(base);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(pipe.empty(s));
@@ -320,31 +357,63 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                                  __fdiv_rn(1.0f, den.w));
             }
         }
-        // ---- the gradient rows, one fill of up to 8 workers at a time
+        // ---- the gradient rows, one fill of up to 8 workers at a time.  Every lane ends up with
+        // all words of every worker; lane k writes worker k of the fill through a pointer it
+        // computes once per fill, and the fill's scales go out as one store.
         uint32_t rmax = 0;
+        constexpr int kWords = 4 * CODEC;
         for (uint32_t m0 = 0; m0 < M; m0 += G::kRows) {
             const uint32_t s = it % G::kStages, use = it / G::kStages;
             if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {
                 atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
                 return;
             }
-            const uint32_t base = pipe.data + s * G::kStageBytes + my;
+            const unsigned char* base = stages + s * G::kStageBytes + my;
+            const uint32_t mine = m0 + (uint32_t)lane;                       // the worker this lane writes
+            uint32_t* my_codes = a.codes + ((uint64_t)mine * a.wpw + T * (uint64_t)kWords);
+            float my_R = 0.0f;
             if (m0 + G::kRows <= M) {
+                // Copy the warp's share of the fill into registers and hand the stage back at once:
+                // the copy engine can refill it while the arithmetic below runs, so loads stay in
+                // flight all the time instead of in bursts at the end of every fill.
+                float4 g[G::kRows];
 #pragma unroll
-                for (int k = 0; k < G::kRows; ++k) {
-                    const float4 g = lds128(base + (uint32_t)k * G::kRowBytes);
-                    rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, q_lo, q_hi, T, lane, 0xFu));
+                for (int k = 0; k < G::kRows; ++k) g[k] = *reinterpret_cast<const float4*>(base + (uint32_t)k * G::kRowBytes);
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pipe.empty(s));
+#pragma unroll
+                for (int k0 = 0; k0 < G::kRows; k0 += kPhiloxBatch) {
+                    uint4 x[kPhiloxBatch];
+                    philox4x32_10_rk_batch<kPhiloxBatch>(q_lo, q_hi, m0 + k0, a.step, a.rk, x);
+#pragma unroll
+                    for (int kk = 0; kk < kPhiloxBatch; ++kk) {
+                        const int k = k0 + kk;
+                        uint32_t w[kWords];
+                        float R;
+                        encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g[k], op, m0 + k, T, x[kk], T, lane, 0xFu, w, R);
+                        store_words_if<CODEC>(lane == k, my_codes, w);
+                        my_R = (lane == k) ? R : my_R;
+                        rmax = max(rmax, __float_as_uint(R));
+                    }
                 }
             } else {
                 for (uint32_t k = 0; m0 + k < M; ++k) {
-                    const float4 g = lds128(base + k * G::kRowBytes);
-                    rmax = max(rmax, encode_worker<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, q_lo, q_hi, T, lane, 0xFu));
+                    const float4 g = *reinterpret_cast<const float4*>(base + k * G::kRowBytes);
+                    uint32_t w[kWords];
+                    float R;
+                    const uint4 x = philox4x32_10_rk(q_lo, q_hi, m0 + k, a.step, a.rk);
+                    encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, x, T, lane, 0xFu, w, R);
+                    store_words_if<CODEC>((uint32_t)lane == k, my_codes, w);
+                    my_R = ((uint32_t)lane == k) ? R : my_R;
+                    rmax = max(rmax, __float_as_uint(R));
                 }
+                __syncwarp();
+                if (lane == 0) mbar_arrive(pipe.empty(s));   // this warp has read the stage
             }
-            __syncwarp();
-            if (lane == 0) mbar_arrive(pipe.empty(s));   // this warp has read the stage
+            if (lane < G::kRows && mine < M) a.scales[(uint64_t)mine * a.nblk + T] = my_R;
             ++it;
         }
+        __syncwarp();
         // NaN or +inf scales are rare: only then count them, from the scales just written
         if (rmax >= 0x7f800000u && lane == 0) {
             unsigned long long bad = 0;

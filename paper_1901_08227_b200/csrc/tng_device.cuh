@@ -47,6 +47,33 @@ __device__ __forceinline__ uint4 philox4x32_10_rk(uint32_t c0, uint32_t c1, uint
     return make_uint4(c0, c1, c2, c3);
 }
 
+// N independent calls that differ only in counter word c2, with their rounds interleaved in
+// program order: the ten rounds of one call form one long dependency chain, N chains side by
+// side keep the pipes busy.
+template <int N>
+__device__ __forceinline__ void philox4x32_10_rk_batch(uint32_t c0, uint32_t c1, uint32_t c2_first, uint32_t c3,
+                                                       const uint32_t (&rk)[20], uint4 (&out)[N]) {
+    uint32_t a0[N], a1[N], a2[N], a3[N];
+#pragma unroll
+    for (int i = 0; i < N; ++i) { a0[i] = c0; a1[i] = c1; a2[i] = c2_first + (uint32_t)i; a3[i] = c3; }
+#pragma unroll
+    for (int round = 0; round < 10; ++round) {
+#pragma unroll
+        for (int i = 0; i < N; ++i) {
+            const uint64_t p0 = static_cast<uint64_t>(kPhiloxMul0) * a0[i];
+            const uint64_t p1 = static_cast<uint64_t>(kPhiloxMul1) * a2[i];
+            const uint32_t n0 = static_cast<uint32_t>(p1 >> 32) ^ a1[i] ^ rk[2 * round];
+            const uint32_t n2 = static_cast<uint32_t>(p0 >> 32) ^ a3[i] ^ rk[2 * round + 1];
+            a1[i] = static_cast<uint32_t>(p1);
+            a3[i] = static_cast<uint32_t>(p0);
+            a0[i] = n0;
+            a2[i] = n2;
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < N; ++i) out[i] = make_uint4(a0[i], a1[i], a2[i], a3[i]);
+}
+
 // u in [0,1) on a 2^-24 grid: the top 24 bits of the word (exact in fp32).
 __device__ __forceinline__ float uniform24(uint32_t x) {
     return __uint2float_rn(x >> 8) * 0x1p-24f;

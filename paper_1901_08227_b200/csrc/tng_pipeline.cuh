@@ -69,6 +69,24 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+// Same for the producer thread, which has nothing else to do: each poll may sleep up to
+// `kProducerNapNs` inside the hardware wait, so that its polling does not take issue slots
+// from the compute warps of its scheduler.  Still bounded.
+constexpr uint32_t kProducerNapNs = 2000;
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity) {
+    for (int i = 0; i < kSpinLimit; ++i) {
+        uint32_t ok;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(ok)
+            : "r"(bar), "r"(parity), "r"(kProducerNapNs)
+            : "memory");
+        if (ok) return true;
+    }
+    return false;
+}
 // One row chunk: global -> this CTA's shared memory, completion counted on `bar`.
 // Both addresses 16-byte aligned, bytes a multiple of 16.
 __device__ __forceinline__ void bulk_load(uint32_t dst_smem, const void* src, uint32_t bytes, uint32_t bar) {
@@ -162,7 +180,7 @@ __device__ __forceinline__ uint32_t pipe_produce(const PipeSmem& p, const PipeRo
             const int n = (seg_end - r0 < G::kRows) ? seg_end - r0 : G::kRows;
             const uint32_t s = it % G::kStages, use = it / G::kStages;
             // a stage is free once its previous use has been consumed (parity of use - 1)
-            if (use > 0 && !mbar_wait(p.empty(s), (use - 1) & 1u)) return kPipeEmptyTimeout;
+            if (use > 0 && !mbar_wait_relaxed(p.empty(s), (use - 1) & 1u)) return kPipeEmptyTimeout;
             mbar_expect_tx(p.full(s), (uint32_t)n * G::kRowBytes);
             const uint32_t dst = p.data + s * G::kStageBytes;
             for (int r = 0; r < n; ++r)
