@@ -70,6 +70,8 @@ def lib():
         L.tngo_quot_den.argtypes = [_f32p, C.c_uint64, C.c_float, _f32p]
         L.tngo_encode.argtypes = [_f32p, C.c_int, C.c_uint64, C.c_uint64, _f32p, C.c_int, C.c_float, C.c_int,
                                   C.c_uint64, C.c_int, C.c_int, C.c_uint32, C.c_uint32, C.c_uint32, _u32p, _f32p]
+        L.tngo_encode_at.argtypes = [_f32p, C.c_int, C.c_uint64, C.c_uint64, _f32p, C.c_int, C.c_float, C.c_int,
+                                     C.c_uint64, C.c_int, C.c_int, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, _u32p, _f32p]
         L.tngo_decode_aggregate.argtypes = [_u32p, _f32p, C.c_int, C.c_uint64, _f32p, C.c_int, C.c_float, C.c_int,
                                             C.c_uint64, C.c_int, _f32p]
         L.tngo_dequant.restype = C.c_float
@@ -217,15 +219,17 @@ def quot_den(ref, quot_eps=2.0 ** -4):
     return den
 
 
-def encode(grads, ref, norm, codec, B=128, s=7, scale_kind=SCALE_ABSMAX, seed=(0, 0), t=0, quot_eps=2.0 ** -4):
-    """Returns (codes[M, words_per_worker] uint32, scales[M, num_blocks] float32)."""
+def encode(grads, ref, norm, codec, B=128, s=7, scale_kind=SCALE_ABSMAX, seed=(0, 0), t=0, quot_eps=2.0 ** -4,
+           coord_offset=0):
+    """Returns (codes[M, words_per_worker] uint32, scales[M, num_blocks] float32).  With
+    coord_offset = i0 the columns handed in are coordinates i0.. of a longer vector."""
     g, M, ld = _rows(grads)
     d = g.shape[1]
     r = None if ref is None else np.ascontiguousarray(ref, dtype=np.float32)
     codes = np.zeros((M, words_per_worker(d, codec)), dtype=np.uint32)
     scales = np.zeros((M, num_blocks(d, B)), dtype=np.float32)
-    lib().tngo_encode(_ptr_f32(g), M, ld, d, _ptr_f32(r), norm, quot_eps, codec, B, s, scale_kind,
-                      seed[0], seed[1], t, codes.ctypes.data_as(_u32p), _ptr_f32(scales))
+    lib().tngo_encode_at(_ptr_f32(g), M, ld, d, _ptr_f32(r), norm, quot_eps, codec, B, s, scale_kind,
+                         seed[0], seed[1], t, int(coord_offset), codes.ctypes.data_as(_u32p), _ptr_f32(scales))
     return codes, scales
 
 

@@ -335,9 +335,11 @@ float tngo_dequant(int codec, int s, uint32_t symbol, float R) {
 /* ------------------------------------------------------------------------- */
 /* encode                                                                     */
 /* ------------------------------------------------------------------------- */
-void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
-                 float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
-                 uint32_t seed_hi, uint32_t t, uint32_t* codes, float* scales) {
+/* The d coordinates handed in are coordinates i0 .. i0+d-1 of a longer vector (i0 a
+ * multiple of the block size and of 128): only the Philox counters see i0. */
+void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
+                    float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
+                    uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales) {
     uint64_t wpw = tngo_words_per_worker(d, codec);
     uint64_t nblk = tngo_num_blocks(d, B);
     uint64_t Beff = (B == 0) ? d : B;
@@ -367,7 +369,7 @@ void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float
         if (!scale_is_bad(R)) {
             uint32_t* codes_m = codes + (uint64_t)m * wpw;
             for (uint64_t i = 0; i < n; ++i) {
-                float u = tngo_coord_uniform(seed_lo, seed_hi, lo + i, (uint32_t)m, t);
+                float u = tngo_coord_uniform(seed_lo, seed_hi, i0 + lo + i, (uint32_t)m, t);
                 uint32_t sym;
                 if (codec == TNGO_CODEC_TERN2) sym = quant_tern2(v[i], R, u);
                 else if (codec == TNGO_CODEC_SIGN1) sym = quant_sign1(v[i], R, u);
@@ -379,6 +381,12 @@ void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float
         free(v);
     }
     free(opnd);
+}
+
+void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
+                 float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
+                 uint32_t seed_hi, uint32_t t, uint32_t* codes, float* scales) {
+    tngo_encode_at(grads, M, ld, d, ref, norm, quot_eps, codec, B, s, scale_kind, seed_lo, seed_hi, t, 0, codes, scales);
 }
 
 /* ------------------------------------------------------------------------- */

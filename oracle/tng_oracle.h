@@ -79,6 +79,12 @@ void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float
                  float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
                  uint32_t seed_hi, uint32_t t, uint32_t* codes, float* scales);
 
+/* Same for a window of a longer vector: the d coordinates are i0 .. i0+d-1 of it (i0 a
+ * multiple of 128 and of B), which only moves the Philox counters. */
+void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
+                    float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
+                    uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales);
+
 /* ---- decode + aggregate + de-normalise (Eq. 2 / Eq. 3, Algorithm 1 "average") */
 void tngo_decode_aggregate(const uint32_t* codes, const float* scales, int M, uint64_t d,
                            const float* ref, int norm, float quot_eps, int codec, uint64_t B,

@@ -1,0 +1,81 @@
+"""GPU parity at the benchmark's full size and launch configuration: d = 2^27 coordinates,
+M = 8 workers, K = 8 ring entries, quotient form, ternary codes, one scale per 128
+coordinates, least-squares fusion -- one whole round through tng_step, as bench.py times it.
+
+The fusion statistics are global sums, so the oracle computes them on the whole vectors; the
+reference, the wire and the aggregate are checked bit for bit on sampled windows of
+coordinates (first and last chunks, windows that straddle chunk boundaries, random ones),
+which the oracle encodes one by one with the window's coordinate offset."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gpu_util import rel_l2, to_np
+from paper_1901_08227_b200 import tng, workloads
+
+pytestmark = pytest.mark.gpu
+
+D, M, K = 1 << 27, 8, 8
+
+
+def test_full_size_round_in_the_benchmark_configuration():
+    free, _ = torch.cuda.mem_get_info()
+    if free < 24 * (1 << 30):
+        pytest.skip("needs about 24 GiB of free device memory")
+    dev = "cuda"
+    stream = workloads.GradientStream(0, D, M, device=dev)
+    ctx = tng.Context(D, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, block=128, fuse_mode=tng.FUSE_LSQ)
+    hist = []                                         # host copies, oldest first
+    for _ in range(K):
+        mu = stream.advance()
+        ctx.push_reference(mu)
+        hist.append(to_np(mu))
+    hist = hist[::-1]                                 # newest first, as the fusion numbers them
+    stream.advance()
+    g = stream.worker_grads()
+    del stream
+    out = torch.empty(D, device=dev)
+    ctx.step(g, out)
+    torch.cuda.synchronize()
+    st = ctx.stats()
+    assert st.pipeline_error == 0 and st.solver_fallback == 0 and st.nonfinite_scales == 0
+    assert st.rounds == 1 and st.k == K
+
+    # ---- fusion statistics and coefficients against the oracle on the whole vectors
+    gn = to_np(g)
+    oG, oc, ogg = oracle.fuse_stats(hist, gn)
+    G = np.array(st.gram[:]).reshape(16, 16)[:K, :K]
+    assert rel_l2(G, oG) < 1e-10
+    assert rel_l2(np.array(st.rhs[:K]), oc) < 1e-6
+    assert st.grad_sq == pytest.approx(ogg, rel=1e-6)
+    a64, a32, flag = oracle.fuse_solve(oG, oc, 1e-6)
+    assert flag == 0
+    alpha = np.array(st.alpha[:K])
+    assert np.allclose(alpha, a64, rtol=0, atol=1e-5 * max(1.0, np.abs(a64).max()))
+    alpha32 = alpha.astype(np.float32)                # what the combine used
+
+    # ---- reference, wire and aggregate on sampled windows, bit for bit
+    ref = ctx.reference()
+    codes, scales = ctx.wire()
+    newest = ctx.history(0)
+    rng = np.random.default_rng(0)
+    windows = [(0, 2048), (D - 2048, 2048), (2048 * 148 - 256, 512), (2048 * 149 * 7 - 128, 256)]
+    windows += [(int(t) * 128, 1024) for t in rng.integers(0, D // 128 - 8, size=60)]
+    for i0, n in windows:
+        sl = slice(i0, i0 + n)
+        want_ref = oracle.combine([h[sl] for h in hist], alpha32)
+        got_ref = to_np(ref[sl])
+        assert np.array_equal(got_ref.view(np.uint32), want_ref.view(np.uint32)), f"reference differs in window {i0}"
+        wc, ws = oracle.encode(np.ascontiguousarray(gn[:, sl]), want_ref, tng.NORM_QUOT, tng.CODEC_TERN2, B=128, seed=(0, 0),
+                               t=0, coord_offset=i0)
+        t0, t1 = i0 // 128, (i0 + n) // 128
+        assert np.array_equal(to_np(codes[:, t0 * 8:t1 * 8]).view(np.uint32), wc), f"codes differ in window {i0}"
+        assert np.array_equal(to_np(scales[:, t0:t1]).view(np.uint32), ws.view(np.uint32)), f"scales differ in window {i0}"
+        want_out = oracle.decode_aggregate(wc, ws, n, want_ref, tng.NORM_QUOT, tng.CODEC_TERN2, B=128)
+        assert np.array_equal(to_np(out[sl]).view(np.uint32), want_out.view(np.uint32)), f"aggregate differs in window {i0}"
+        assert np.array_equal(to_np(newest[sl]).view(np.uint32), want_out.view(np.uint32))
+    # ---- properties that hold at any size
+    assert bool(torch.isfinite(out).all())
+    assert bool((scales >= 0).all())
+    ctx.close()

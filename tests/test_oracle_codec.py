@@ -411,3 +411,23 @@ def test_cnz_of_proposition_2():
     r = g.mean(0)
     want = ((g.astype(np.float64) - r.astype(np.float64)) ** 2).sum() / (g.astype(np.float64) ** 2).sum()
     assert oracle.cnz(g, r) == pytest.approx(want, rel=1e-12)
+
+
+@pytest.mark.parametrize("codec", [oracle.CODEC_SIGN1, oracle.CODEC_TERN2, oracle.CODEC_QSGD4])
+def test_encoding_a_window_equals_the_window_of_the_whole_encode(codec):
+    # coordinates [i0, i0+n) encoded with coord_offset = i0 give exactly the words and scales the
+    # whole-vector encode has for those tiles (tiles are independent given the reference)
+    d, M, i0, n = 128 * 40 + 17, 3, 128 * 13, 128 * 9
+    rng = np.random.default_rng(5)
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    r = (0.8 * g.mean(0) + 0.1 * rng.standard_normal(d)).astype(np.float32)
+    for norm in (oracle.NORM_DIFF, oracle.NORM_QUOT):
+        codes, scales = oracle.encode(g, r, norm, codec, B=128, s=5, seed=(7, 1), t=3)
+        wc, ws = oracle.encode(np.ascontiguousarray(g[:, i0:i0 + n]), r[i0:i0 + n], norm, codec, B=128, s=5, seed=(7, 1), t=3,
+                               coord_offset=i0)
+        words = 4 * codec
+        assert np.array_equal(wc, codes[:, i0 // 128 * words:(i0 + n) // 128 * words])
+        assert np.array_equal(ws.view(np.uint32), scales[:, i0 // 128:(i0 + n) // 128].view(np.uint32))
+        # and without the offset the random draws differ
+        wc0, _ = oracle.encode(np.ascontiguousarray(g[:, i0:i0 + n]), r[i0:i0 + n], norm, codec, B=128, s=5, seed=(7, 1), t=3)
+        assert not np.array_equal(wc0, wc)
