@@ -144,6 +144,21 @@ def config_dict(name, cfg, world):
             "sharding": "one process per GPU, each rank its own d coordinates" if world > 1 else "single GPU"}
 
 
+def max_over_ranks(value, world, device):
+    """The slowest rank's time: every rank gets max_r value_r (the job is as slow as that rank)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([float(value)], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.item()
+
+
+def job_throughput_gbs(world, M, d, seconds_per_step):
+    """GB/s of fp32 gradient of the whole job: every rank pushes its own M x d problem per step."""
+    return world * M * d * 4 / seconds_per_step / 1e9
+
+
 # --------------------------------------------------------------------------------------
 def run_reference(args, name, cfg):
     """The CPU oracle, as it stands, timed on a bounded sample of the workload."""
@@ -266,11 +281,7 @@ def run_ours(args, name, cfg):
     ev1.record()
     barrier()
     clocks = sampler.stop()
-    ms_total = ev0.elapsed_time(ev1)
-    t = torch.tensor([ms_total], dtype=torch.float64, device=dev)
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step = t.item() / args.steps
+    ms_step = max_over_ranks(ev0.elapsed_time(ev1), world, dev) / args.steps
     st1 = ctx.stats()
     launches = st1.kernel_launches - st0.kernel_launches
 
@@ -317,17 +328,15 @@ def run_ours(args, name, cfg):
         for _ in range(e2e_steps):
             ctx_h.step_host(g_host, o_host)
         torch.cuda.synchronize()
-        dt = torch.tensor([(time.perf_counter() - t0) / e2e_steps], dtype=torch.float64, device=dev)
-        if world > 1:
-            dist.all_reduce(dt, op=dist.ReduceOp.MAX)
-        e2e = {"value": world * M * d * 4 / dt.item() / 1e9, "unit": UNIT, "h2d_bytes_per_step": M * d * 4,
-               "d2h_bytes_per_step": d * 4, "steps": e2e_steps, "ms_per_step": dt.item() * 1e3,
+        dt = max_over_ranks((time.perf_counter() - t0) / e2e_steps, world, dev)
+        e2e = {"value": job_throughput_gbs(world, M, d, dt), "unit": UNIT, "h2d_bytes_per_step": M * d * 4,
+               "d2h_bytes_per_step": d * 4, "steps": e2e_steps, "ms_per_step": dt * 1e3,
                "api": "tng_step_host (pinned host rows -> device staging -> round -> aggregate back to host)"}
         ctx_h.close()
         del g_host, o_host
 
     if rank == 0:
-        value = world * M * d * 4 / (ms_step * 1e-3) / 1e9
+        value = job_throughput_gbs(world, M, d, ms_step * 1e-3)
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
