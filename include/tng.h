@@ -68,7 +68,11 @@ typedef enum {
     TNG_OPT_RIDGE = 6,       /* relative ridge of the K x K solve.  Default 1e-6. */
     TNG_OPT_QUOT_EPS = 7,    /* floor of |r| relative to its tile maximum, quotient form.  Default 2^-4. */
     TNG_OPT_TIMING = 8,      /* 1 = record CUDA events around every stage of tng_step.  Default 0. */
-    TNG_OPT_HOST_STAGING = 9 /* 1 = reserve device staging so tng_step_host can be used.  Default 0. */
+    TNG_OPT_HOST_STAGING = 9,/* 1 = reserve device staging so tng_step_host can be used.  Default 0. */
+    TNG_OPT_REF_EVERY = 10   /* refresh cadence of the reference (Sec. 3.1, last paragraph; Sec. 4.1 refreshes
+                                every 16 iterations): tng_step fuses a new reference in rounds t with
+                                t % value == 0 and reuses the previous one in between; the ring still
+                                receives every aggregate.  1..65536, default 1. */
 } tng_option;
 
 #define TNG_MAX_WORKERS 64
@@ -129,7 +133,22 @@ tng_status tng_step(tng_ctx* ctx, const float* grads_dev, uint64_t ld, float* ag
 tng_status tng_step_host(tng_ctx* ctx, const float* grads_host, uint64_t ld, float* agg_out_host,
                          void* stream);
 
-/* ---- stage-level entry points (the same kernels tng_step launches) ---------- */
+/* ---- state save / resume ----------------------------------------------------- */
+/* The state a context carries between rounds is the ring, the round counter and (with a refresh
+ * cadence above 1) the held reference; the codes of round t depend on nothing else, so a context
+ * that loads a saved state continues bit for bit.  The blob lives in HOST memory.
+ * tng_state_bytes: upper bound of the blob for this context.
+ * tng_save_state:  waits for `stream`, writes the blob to host_buf (capacity `bytes`), returns the
+ *                  bytes used in *written (may be NULL).  TNG_ERR_ALLOC if the buffer is too small.
+ * tng_load_state:  the context must have been created with the same d, M, K, codec, normalisation
+ *                  and options (else TNG_ERR_INVALID_ARG); replaces ring, counter and reference;
+ *                  returns after the copies have finished. */
+tng_status tng_state_bytes(tng_ctx* ctx, size_t* bytes);
+tng_status tng_save_state(tng_ctx* ctx, void* host_buf, size_t bytes, size_t* written, void* stream);
+tng_status tng_load_state(tng_ctx* ctx, const void* host_buf, size_t bytes, void* stream);
+
+/* ---- stage-level entry points (the kernels tng_step launches; tng_step itself folds the
+ * reference combine into the encode pass when there is one scale per 128 coordinates) ---------- */
 /* Fusion: Gram/rhs statistics, K x K solve, reference combine -> the context's reference. */
 tng_status tng_fuse(tng_ctx* ctx, const float* grads_dev, uint64_t ld, void* stream);
 /* Normalise + scale + quantise + pack against ref_dev (NULL = the context's reference).

@@ -27,7 +27,7 @@ CODEC_SIGN1, CODEC_TERN2, CODEC_QSGD4 = 1, 2, 4
 NORM_NONE, NORM_DIFF, NORM_QUOT = 0, 1, 2
 SCALE_ABSMAX, SCALE_L2 = 0, 1
 FUSE_AUTO, FUSE_LAST, FUSE_MEAN, FUSE_LSQ, FUSE_HINDSIGHT = 0, 1, 2, 3, 4
-OPT_BLOCK, OPT_QSGD_LEVELS, OPT_SCALE_KIND, OPT_SEED_LO, OPT_SEED_HI, OPT_FUSE_MODE, OPT_RIDGE, OPT_QUOT_EPS = range(8)
+OPT_BLOCK, OPT_QSGD_LEVELS, OPT_SCALE_KIND, OPT_SEED_LO, OPT_SEED_HI, OPT_FUSE_MODE, OPT_RIDGE, OPT_QUOT_EPS, OPT_REF_EVERY = range(9)
 TILE = 128
 
 
@@ -269,7 +269,7 @@ class State:
         self.B = 128
         names = {"block": OPT_BLOCK, "qsgd_levels": OPT_QSGD_LEVELS, "scale_kind": OPT_SCALE_KIND,
                  "seed_lo": OPT_SEED_LO, "seed_hi": OPT_SEED_HI, "fuse_mode": OPT_FUSE_MODE,
-                 "ridge": OPT_RIDGE, "quot_eps": OPT_QUOT_EPS}
+                 "ridge": OPT_RIDGE, "quot_eps": OPT_QUOT_EPS, "ref_every": OPT_REF_EVERY}
         for key, val in options.items():
             if lib().tngo_set_option(self._h, names[key], float(val)):
                 raise ValueError(f"bad option {key}={val}")

@@ -451,6 +451,7 @@ struct tngo_state {
     int M, K, codec, norm;
     uint64_t B;
     int s, scale_kind, fuse_mode;
+    uint32_t ref_every; /* the reference is re-fused in rounds t with t % ref_every == 0 */
     uint32_t seed_lo, seed_hi;
     double ridge;
     float quot_eps;
@@ -474,7 +475,7 @@ tngo_state* tngo_create(uint64_t d, int M, int K, int codec, int norm) {
     tngo_state* st = (tngo_state*)calloc(1, sizeof *st);
     st->d = d; st->M = M; st->K = K; st->codec = codec; st->norm = norm;
     st->B = 128; st->s = 7; st->scale_kind = TNGO_SCALE_ABSMAX; st->fuse_mode = 0;
-    st->seed_lo = 0; st->seed_hi = 0; st->ridge = 1e-6; st->quot_eps = 0x1p-4f;
+    st->seed_lo = 0; st->seed_hi = 0; st->ridge = 1e-6; st->quot_eps = 0x1p-4f; st->ref_every = 1;
     st->H = (float*)calloc((size_t)K * d, sizeof(float));
     st->ref = (float*)calloc(d, sizeof(float));
     st->codes = (uint32_t*)calloc((size_t)M * tngo_words_per_worker(d, codec), sizeof(uint32_t));
@@ -511,6 +512,9 @@ int tngo_set_option(tngo_state* st, int key, double value) {
         case 7:
             if (!(value > 0 && value <= 1)) return 1;
             st->quot_eps = (float)value; return 0;
+        case 8:
+            if (value < 1 || value > 65536) return 1;
+            st->ref_every = (uint32_t)value; return 0;
         default: return 1;
     }
 }
@@ -573,8 +577,10 @@ void tngo_stage_decode_push(tngo_state* st, float* out) {
     st->t += 1;
 }
 
+/* Reference refresh cadence (Sec. 3.1, last paragraph): a new reference only in rounds t with
+ * t % ref_every == 0; in between the previous one is kept.  The ring receives every aggregate. */
 void tngo_step(tngo_state* st, const float* grads, uint64_t ld, float* out) {
-    tngo_stage_fuse(st, grads, ld);
+    if (st->t % st->ref_every == 0) tngo_stage_fuse(st, grads, ld);
     tngo_stage_encode(st, grads, ld);
     tngo_stage_decode_push(st, out);
 }

@@ -102,7 +102,7 @@ typedef struct tngo_state tngo_state;
 tngo_state* tngo_create(uint64_t d, int M, int K, int codec, int norm);
 void tngo_destroy(tngo_state* st);
 /* keys: 0 block, 1 qsgd levels, 2 scale kind, 3 seed lo, 4 seed hi, 5 fuse mode
- * (0 auto), 6 ridge, 7 quot eps.  Returns 0 ok, nonzero on a bad key/value. */
+ * (0 auto), 6 ridge, 7 quot eps, 8 reference refresh cadence (tngo_step only).  Returns 0 ok, nonzero on a bad key/value. */
 int tngo_set_option(tngo_state* st, int key, double value);
 void tngo_push_reference(tngo_state* st, const float* vec);
 /* One round: fuse -> normalise -> encode -> decode -> aggregate -> push. */

@@ -27,6 +27,7 @@ struct tng_ctx {
     // options
     uint64_t block_opt = 128;
     int levels = 7, scale_kind = 0, fuse_mode = TNG_FUSE_AUTO, timing = 0, host_staging = 0;
+    uint32_t ref_every = 1;
     uint32_t seed_lo = 0, seed_hi = 0;
     double ridge = 1e-6;
     float quot_eps = 0.0625f;
@@ -256,8 +257,19 @@ tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, c
 tng_status step_impl(tng_ctx* c, const float* grads, uint64_t ld, float* out, cudaStream_t st) {
     StageTimer tm(c, st);
     RefFusion fusion;
-    tng_status s = do_fuse(c, grads, ld, st, &tm, &fusion);
-    if (s != TNG_OK) return s;
+    fusion.k = 0;
+    tng_status s = TNG_OK;
+    if (c->rounds % c->ref_every == 0 || !c->ref_cur) {
+        s = do_fuse(c, grads, ld, st, &tm, &fusion);
+        if (s != TNG_OK) return s;
+        if (c->ref_every > 1 && c->ref_cur != c->ref_buf()) {
+            // the reference is held for several rounds: it must not alias a ring slot that will be overwritten
+            TNG_CUDA(c, cudaMemcpyAsync(c->ref_buf(), c->ref_cur, c->d * sizeof(float), cudaMemcpyDeviceToDevice, st));
+            c->ref_cur = c->ref_buf();
+        }
+    } else {   // between refreshes: the held reference, no fusion pass
+        tm.mark(0, false); tm.mark(1, false); tm.mark(2, false);
+    }
     s = do_encode(c, grads, ld, c->ref_cur, &fusion, (uint32_t)c->rounds, st);
     if (s != TNG_OK) return s;
     tm.mark(3, true);
@@ -333,6 +345,9 @@ tng_status tng_set_option(tng_ctx* c, tng_option key, double value) {
         case TNG_OPT_HOST_STAGING:
             if (value != 0 && value != 1) return TNG_ERR_INVALID_ARG;
             c->host_staging = (int)value; return TNG_OK;
+        case TNG_OPT_REF_EVERY:
+            if (value < 1 || value > 65536 || value != floor(value)) return TNG_ERR_INVALID_ARG;
+            c->ref_every = (uint32_t)value; return TNG_OK;
         default: return TNG_ERR_INVALID_ARG;
     }
 }
@@ -390,6 +405,91 @@ tng_status tng_step_host(tng_ctx* c, const float* grads_host, uint64_t ld, float
     if (s != TNG_OK) return s;
     TNG_CUDA(c, cudaMemcpyAsync(agg_out_host, c->stage_o(), c->d * sizeof(float), cudaMemcpyDeviceToHost, st));
     TNG_CUDA(c, cudaStreamSynchronize(st));
+    return TNG_OK;
+}
+
+namespace {
+struct StateHeader {
+    uint32_t magic, version;
+    uint64_t d;
+    uint32_t M, K, codec, norm;
+    uint64_t block;
+    uint32_t levels, scale_kind, fuse_mode, seed_lo, seed_hi, ref_every;
+    double ridge;
+    float quot_eps;
+    uint32_t k;
+    uint64_t rounds;
+    uint32_t has_ref, pad;
+};
+constexpr uint32_t kStateMagic = 0x53474e54u;   // "TNGS"
+
+void fill_header(const tng_ctx* c, StateHeader* h) {
+    memset(h, 0, sizeof *h);
+    h->magic = kStateMagic; h->version = 1;
+    h->d = c->d; h->M = c->M; h->K = c->K; h->codec = (uint32_t)c->codec; h->norm = (uint32_t)c->norm;
+    h->block = c->block_opt; h->levels = (uint32_t)c->levels; h->scale_kind = (uint32_t)c->scale_kind;
+    h->fuse_mode = (uint32_t)c->fuse_mode; h->seed_lo = c->seed_lo; h->seed_hi = c->seed_hi; h->ref_every = c->ref_every;
+    h->ridge = c->ridge; h->quot_eps = c->quot_eps;
+    h->k = c->k; h->rounds = c->rounds; h->has_ref = 0;
+}
+}  // namespace
+
+tng_status tng_state_bytes(tng_ctx* c, size_t* bytes) {
+    if (!c || !bytes) return TNG_ERR_INVALID_ARG;
+    *bytes = sizeof(StateHeader) + ((size_t)c->K + 1) * c->d * sizeof(float);
+    return TNG_OK;
+}
+
+tng_status tng_save_state(tng_ctx* c, void* host_buf, size_t bytes, size_t* written, void* stream) {
+    if (!c || !host_buf) return TNG_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    StateHeader h;
+    fill_header(c, &h);
+    h.has_ref = (c->ref_every > 1 && c->ref_cur) ? 1u : 0u;
+    const size_t vec = c->d * sizeof(float);
+    const size_t need = sizeof h + ((size_t)c->k + h.has_ref) * vec;
+    if (bytes < need) return TNG_ERR_ALLOC;
+    char* p = static_cast<char*>(host_buf);
+    memcpy(p, &h, sizeof h);
+    p += sizeof h;
+    for (uint32_t j = 0; j < c->k; ++j, p += vec)   // newest first
+        TNG_CUDA(c, cudaMemcpyAsync(p, c->ring(c->hist_slot(j)), vec, cudaMemcpyDeviceToHost, st));
+    if (h.has_ref) TNG_CUDA(c, cudaMemcpyAsync(p, c->ref_cur, vec, cudaMemcpyDeviceToHost, st));
+    TNG_CUDA(c, cudaStreamSynchronize(st));
+    if (written) *written = need;
+    return TNG_OK;
+}
+
+tng_status tng_load_state(tng_ctx* c, const void* host_buf, size_t bytes, void* stream) {
+    if (!c || !host_buf || bytes < sizeof(StateHeader)) return TNG_ERR_INVALID_ARG;
+    StateHeader h, mine;
+    memcpy(&h, host_buf, sizeof h);
+    fill_header(c, &mine);
+    if (h.magic != kStateMagic || h.version != 1 || h.d != mine.d || h.M != mine.M || h.K != mine.K || h.codec != mine.codec ||
+        h.norm != mine.norm || h.block != mine.block || h.levels != mine.levels || h.scale_kind != mine.scale_kind ||
+        h.fuse_mode != mine.fuse_mode || h.seed_lo != mine.seed_lo || h.seed_hi != mine.seed_hi || h.ref_every != mine.ref_every ||
+        h.ridge != mine.ridge || h.quot_eps != mine.quot_eps || h.k > h.K || h.has_ref > 1)
+        return TNG_ERR_INVALID_ARG;
+    const size_t vec = c->d * sizeof(float);
+    if (bytes < sizeof h + ((size_t)h.k + h.has_ref) * vec) return TNG_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    const char* p = static_cast<const char*>(host_buf) + sizeof h;
+    // h_{j+1} goes to slot k-1-j, the newest entry sitting at head = k-1
+    for (uint32_t j = 0; j < h.k; ++j, p += vec)
+        TNG_CUDA(c, cudaMemcpyAsync(c->ring((int)(h.k - 1 - j)), p, vec, cudaMemcpyHostToDevice, st));
+    if (h.has_ref) TNG_CUDA(c, cudaMemcpyAsync(c->ref_buf(), p, vec, cudaMemcpyHostToDevice, st));
+    TNG_CUDA(c, cudaStreamSynchronize(st));
+    c->k = h.k;
+    c->head = h.k ? (int)h.k - 1 : 0;
+    c->rounds = h.rounds;
+    c->ref_cur = h.has_ref ? c->ref_buf() : nullptr;
+    c->last_mode = c->effective_mode();
+    c->last_had_stats = false;
+    c->last_solved = false;
     return TNG_OK;
 }
 

@@ -15,7 +15,7 @@ NORM_NONE, NORM_DIFF, NORM_QUOT = 0, 1, 2
 SCALE_ABSMAX, SCALE_L2 = 0, 1
 FUSE_AUTO, FUSE_LAST, FUSE_MEAN, FUSE_LSQ, FUSE_HINDSIGHT = 0, 1, 2, 3, 4
 (OPT_BLOCK, OPT_QSGD_LEVELS, OPT_SCALE_KIND, OPT_SEED_LO, OPT_SEED_HI, OPT_FUSE_MODE, OPT_RIDGE, OPT_QUOT_EPS,
- OPT_TIMING, OPT_HOST_STAGING) = range(10)
+ OPT_TIMING, OPT_HOST_STAGING, OPT_REF_EVERY) = range(11)
 (OK, ERR_INVALID_ARG, ERR_STATE, ERR_ALLOC, ERR_CUDA, ERR_NONFINITE, ERR_UNSUPPORTED) = range(7)
 MAX_HISTORY = 16
 TILE = 128
@@ -26,7 +26,7 @@ EXPORTS = [
     "tng_push_reference", "tng_step", "tng_step_host", "tng_fuse", "tng_encode", "tng_decode_aggregate",
     "tng_wire", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
     "tng_logistic_scratch_floats", "tng_logistic_grad", "tng_logistic_loss", "tng_rosenbrock_grad",
-    "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static",
+    "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static", "tng_state_bytes", "tng_save_state", "tng_load_state",
 ]
 
 
@@ -86,6 +86,9 @@ def lib():
         L.tng_rosenbrock_grad.argtypes = [vp, u64, vp, u32, u64, vp, vp]
         L.tng_rosenbrock_value.argtypes = [vp, u64, vp, vp]
         L.tng_sgd_update.argtypes = [vp, vp, u64, f32, vp]
+        L.tng_state_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
+        L.tng_save_state.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t), vp]
+        L.tng_load_state.argtypes = [vp, vp, C.c_size_t, vp]
         L.tng_gram_static.argtypes = [C.POINTER(vp), u32, u64, vp, u32, u64, vp, vp]
         _lib = L
     return _lib
@@ -126,7 +129,7 @@ class Context:
 
     _OPTS = {"block": OPT_BLOCK, "qsgd_levels": OPT_QSGD_LEVELS, "scale_kind": OPT_SCALE_KIND,
              "seed_lo": OPT_SEED_LO, "seed_hi": OPT_SEED_HI, "fuse_mode": OPT_FUSE_MODE, "ridge": OPT_RIDGE,
-             "quot_eps": OPT_QUOT_EPS, "timing": OPT_TIMING, "host_staging": OPT_HOST_STAGING}
+             "quot_eps": OPT_QUOT_EPS, "timing": OPT_TIMING, "host_staging": OPT_HOST_STAGING, "ref_every": OPT_REF_EVERY}
 
     def __init__(self, d, M, K, codec, norm, workspace=None, **options):
         self.d, self.M, self.K, self.codec, self.norm = int(d), int(M), int(K), int(codec), int(norm)
@@ -182,6 +185,23 @@ class Context:
         _check(lib().tng_step_host(self._h, grads_host.data_ptr(), grads_host.stride(0), out_host.data_ptr(), _stream()),
                "tng_step_host")
         return out_host
+
+    def state_bytes(self) -> int:
+        n = C.c_size_t()
+        _check(lib().tng_state_bytes(self._h, C.byref(n)), "tng_state_bytes")
+        return n.value
+
+    def save_state(self) -> torch.Tensor:
+        """The context's state (ring, round counter, held reference) as a host byte tensor."""
+        buf = torch.empty(self.state_bytes(), dtype=torch.uint8)
+        used = C.c_size_t()
+        _check(lib().tng_save_state(self._h, buf.data_ptr(), buf.numel(), C.byref(used), _stream()), "tng_save_state")
+        return buf[: used.value].clone()
+
+    def load_state(self, buf: torch.Tensor):
+        if buf.is_cuda or buf.dtype != torch.uint8 or not buf.is_contiguous():
+            raise TypeError("state must be a contiguous host uint8 tensor")
+        _check(lib().tng_load_state(self._h, buf.data_ptr(), buf.numel(), _stream()), "tng_load_state")
 
     def fuse(self, grads):
         p, ld = _rows(grads)

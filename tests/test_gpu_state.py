@@ -1,0 +1,76 @@
+"""GPU: reference refresh cadence (tng_step with TNG_OPT_REF_EVERY) against the oracle, and
+state save / resume (a context that loads a saved state continues bit for bit)."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import codes_np, drifting_grads, make_ctx, make_oracle, same_values, to_np
+from paper_1901_08227_b200 import tng
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("mode,K", [(tng.FUSE_LAST, 1), (tng.FUSE_LAST, 3), (tng.FUSE_MEAN, 4)])
+@pytest.mark.parametrize("norm,codec,B,d", [(tng.NORM_DIFF, tng.CODEC_TERN2, 128, 128 * 9 + 40),
+                                            (tng.NORM_QUOT, tng.CODEC_TERN2, 128, 2048 * 9 + 128 * 3 + 8),
+                                            (tng.NORM_DIFF, tng.CODEC_QSGD4, 256, 3000)])
+def test_refresh_cadence_matches_the_oracle_bit_for_bit(mode, K, norm, codec, B, d):
+    M, steps, tau = 4, 9, 3
+    opts = dict(block=B, fuse_mode=mode, seed_lo=2, qsgd_levels=4, ref_every=tau)
+    ctx = make_ctx(d, M, K, codec, norm, **opts)
+    orc = make_oracle(d, M, K, codec, norm, **opts)
+    out = torch.empty(d, device="cuda")
+    for t, g in enumerate(drifting_grads(31, steps, M, d, "cuda")):
+        ctx.step(g, out)
+        want = orc.step(to_np(g))
+        codes, scales = ctx.wire()
+        assert same_values(to_np(ctx.reference()), orc.ref()), f"reference differs at round {t}"
+        assert np.array_equal(codes_np(codes), orc.codes()), f"codes differ at round {t}"
+        assert same_values(to_np(scales), orc.scales())
+        assert same_values(to_np(out), want)
+    st = ctx.stats()
+    assert st.rounds == steps and st.pipeline_error == 0
+
+
+@pytest.mark.parametrize("mode,tau", [(tng.FUSE_LSQ, 1), (tng.FUSE_LSQ, 4), (tng.FUSE_LAST, 1), (tng.FUSE_MEAN, 2)])
+def test_a_loaded_state_continues_bit_for_bit(mode, tau):
+    d, M, K = 2048 * 9 + 128 * 3 + 8, 5, 3
+    opts = dict(block=128, fuse_mode=mode, seed_lo=7, seed_hi=1, ref_every=tau)
+    a = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, **opts)
+    grads = list(drifting_grads(8, 11, M, d, "cuda"))
+    out = torch.empty(d, device="cuda")
+    for g in grads[:6]:
+        a.step(g, out)
+    blob = a.save_state()
+    assert blob.numel() <= a.state_bytes()
+    tail_a = []
+    for g in grads[6:]:
+        a.step(g, out)
+        tail_a.append((a.wire()[0].clone(), a.wire()[1].clone(), out.clone()))
+    b = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, **opts)
+    b.load_state(blob)
+    assert b.stats().rounds == 6 and b.stats().k == K
+    for g, (codes, scales, o) in zip(grads[6:], tail_a):
+        b.step(g, out)
+        assert torch.equal(b.wire()[0], codes) and torch.equal(b.wire()[1], scales) and torch.equal(out, o)
+    for j in range(K):
+        assert torch.equal(a.history(j), b.history(j))
+
+
+def test_a_state_of_another_configuration_is_rejected():
+    a = make_ctx(1000, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=1)
+    g = torch.randn(2, 1000, device="cuda")
+    a.step(g)
+    blob = a.save_state()
+    for other in (make_ctx(1000, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=2),
+                  make_ctx(1000, 2, 3, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=1),
+                  make_ctx(1004, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=1)):
+        with pytest.raises(tng.TngError) as e:
+            other.load_state(blob)
+        assert e.value.status == tng.ERR_INVALID_ARG
+    with pytest.raises(tng.TngError) as e:
+        a.load_state(blob[:40].clone())
+    assert e.value.status == tng.ERR_INVALID_ARG
+    small = torch.empty(64, dtype=torch.uint8)
+    st = tng.lib().tng_save_state(a._h, small.data_ptr(), small.numel(), None, 0)
+    assert st == tng.ERR_ALLOC

@@ -117,3 +117,26 @@ def test_options_are_validated():
         oracle.State(100, 1, 17, CODEC_TERN2, NORM_DIFF)
     with pytest.raises(ValueError):
         oracle.State(100, 1, 1, 3, NORM_DIFF)
+
+
+def test_reference_refresh_cadence_keeps_the_reference_between_refreshes():
+    # Sec. 3.1 (last paragraph) / Sec. 4.1: the reference may be refreshed only every tau rounds.
+    # With tau = 3 and the delayed-gradient reference, rounds 3..5 all use the aggregate of round 2.
+    d, M, K, tau = 300, 3, 2, 3
+    rng = np.random.default_rng(2)
+    st = oracle.State(d, M, K, oracle.CODEC_TERN2, oracle.NORM_DIFF, fuse_mode=oracle.FUSE_LAST, ref_every=tau, seed_lo=4)
+    every = oracle.State(d, M, K, oracle.CODEC_TERN2, oracle.NORM_DIFF, fuse_mode=oracle.FUSE_LAST, ref_every=1, seed_lo=4)
+    plain = oracle.State(d, M, K, oracle.CODEC_TERN2, oracle.NORM_DIFF, fuse_mode=oracle.FUSE_LAST, seed_lo=4)
+    outs, refs = [], []
+    for t in range(8):
+        g = rng.standard_normal((M, d)).astype(np.float32)
+        outs.append(st.step(g))
+        refs.append(st.ref())
+        assert np.array_equal(every.step(g), plain.step(g))          # tau = 1 is the default behaviour
+    assert not refs[0].any() and not refs[1].any() and not refs[2].any()   # empty ring at the first refresh
+    for t in (3, 4, 5):
+        assert np.array_equal(refs[t], outs[2])                      # refreshed at t = 3 from the newest aggregate
+    for t in (6, 7):
+        assert np.array_equal(refs[t], outs[5])
+    assert st.k == K and st.t == 8                                   # the ring still took every aggregate
+    assert np.array_equal(st.history(0), outs[7]) and np.array_equal(st.history(1), outs[6])
