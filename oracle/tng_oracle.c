@@ -263,6 +263,24 @@ static float normalise(float g, int norm, float r_or_rden) {
     if (norm == TNGO_NORM_QUOT) return g * r_or_rden;
     return g;
 }
+/* Combined form of Section 3 (the unnumbered display after Eq. 3): v = (g - r) ./ r', taken as
+ * one fp32 subtraction and one multiply by the reciprocal of the guarded second reference. */
+static float normalise_comb(float g, float r, float rden2) {
+    float diff = g - r;
+    return diff * rden2;
+}
+
+/* Second reference of the combined form: the per-coordinate magnitude of the trajectory,
+ * r'_d = (1/k) sum_j |h_j,d| as an fp32 fma chain (j ascending, 1/k one IEEE division). */
+void tngo_magnitude_reference(const float* const* h, int k, uint64_t d, float* ref2) {
+    float inv = (k > 0) ? 1.0f / (float)k : 0.0f;
+#pragma omp parallel for
+    for (uint64_t i = 0; i < d; ++i) {
+        float acc = 0.0f;
+        for (int j = 0; j < k; ++j) acc = fmaf(inv, fabsf(h[j][i]), acc);
+        ref2[i] = acc;
+    }
+}
 
 /* ------------------------------------------------------------------------- */
 /* scale of one block                                                         */
@@ -337,8 +355,8 @@ float tngo_dequant(int codec, int s, uint32_t symbol, float R) {
 /* ------------------------------------------------------------------------- */
 /* The d coordinates handed in are coordinates i0 .. i0+d-1 of a longer vector (i0 a
  * multiple of the block size and of 128): only the Philox counters see i0. */
-void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
-                    float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
+void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, const float* ref2,
+                    int norm, float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
                     uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales) {
     uint64_t wpw = tngo_words_per_worker(d, codec);
     uint64_t nblk = tngo_num_blocks(d, B);
@@ -347,8 +365,8 @@ void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const fl
 
     /* per-coordinate operand of the normalisation, shared by all workers */
     float* opnd = (float*)malloc(sizeof(float) * (d ? d : 1));
-    if (norm == TNGO_NORM_QUOT) {
-        tngo_quot_den(ref, d, quot_eps, opnd);
+    if (norm == TNGO_NORM_QUOT || norm == TNGO_NORM_COMB) {
+        tngo_quot_den(norm == TNGO_NORM_QUOT ? ref : ref2, d, quot_eps, opnd);
         for (uint64_t i = 0; i < d; ++i) opnd[i] = 1.0f / opnd[i];
     } else {
         for (uint64_t i = 0; i < d; ++i) opnd[i] = (norm == TNGO_NORM_DIFF && ref) ? ref[i] : 0.0f;
@@ -363,7 +381,9 @@ void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const fl
         uint64_t n = hi - lo;
         const float* g = grads + (uint64_t)m * ld;
         float* v = (float*)malloc(sizeof(float) * (n ? n : 1));
-        for (uint64_t i = 0; i < n; ++i) v[i] = normalise(g[lo + i], norm, opnd[lo + i]);
+        for (uint64_t i = 0; i < n; ++i)
+            v[i] = (norm == TNGO_NORM_COMB) ? normalise_comb(g[lo + i], ref ? ref[lo + i] : 0.0f, opnd[lo + i])
+                                            : normalise(g[lo + i], norm, opnd[lo + i]);
         float R = (scale_kind == TNGO_SCALE_L2) ? l2_scale(v, n) : absmax_nan(v, n);
         scales[(uint64_t)m * nblk + blk] = R;
         if (!scale_is_bad(R)) {
@@ -386,22 +406,22 @@ void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const fl
 void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
                  float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
                  uint32_t seed_hi, uint32_t t, uint32_t* codes, float* scales) {
-    tngo_encode_at(grads, M, ld, d, ref, norm, quot_eps, codec, B, s, scale_kind, seed_lo, seed_hi, t, 0, codes, scales);
+    tngo_encode_at(grads, M, ld, d, ref, NULL, norm, quot_eps, codec, B, s, scale_kind, seed_lo, seed_hi, t, 0, codes, scales);
 }
 
 /* ------------------------------------------------------------------------- */
 /* decode + aggregate + de-normalise                                          */
 /* ------------------------------------------------------------------------- */
-void tngo_decode_aggregate(const uint32_t* codes, const float* scales, int M, uint64_t d,
-                           const float* ref, int norm, float quot_eps, int codec, uint64_t B,
-                           int s, float* out) {
+void tngo_decode_aggregate2(const uint32_t* codes, const float* scales, int M, uint64_t d,
+                            const float* ref, const float* ref2, int norm, float quot_eps, int codec,
+                            uint64_t B, int s, float* out) {
     uint64_t wpw = tngo_words_per_worker(d, codec);
     uint64_t nblk = tngo_num_blocks(d, B);
     uint64_t Beff = (B == 0) ? d : B;
     float* den = NULL;
-    if (norm == TNGO_NORM_QUOT) {
+    if (norm == TNGO_NORM_QUOT || norm == TNGO_NORM_COMB) {
         den = (float*)malloc(sizeof(float) * (d ? d : 1));
-        tngo_quot_den(ref, d, quot_eps, den);
+        tngo_quot_den(norm == TNGO_NORM_QUOT ? ref : ref2, d, quot_eps, den);
     }
 #pragma omp parallel for
     for (uint64_t i = 0; i < d; ++i) {
@@ -418,9 +438,18 @@ void tngo_decode_aggregate(const uint32_t* codes, const float* scales, int M, ui
         float r = (ref ? ref[i] : 0.0f);
         if (norm == TNGO_NORM_DIFF) out[i] = r + a;         /* v = ref + r(w_t), Eq. 2 */
         else if (norm == TNGO_NORM_QUOT) out[i] = den[i] * a; /* v = ref . r(w_t), Eq. 3 */
-        else out[i] = a;
+        else if (norm == TNGO_NORM_COMB) {                    /* v = ref' . r(w_t) + ref */
+            float scaled = den[i] * a;
+            out[i] = scaled + r;
+        } else out[i] = a;
     }
     free(den);
+}
+
+void tngo_decode_aggregate(const uint32_t* codes, const float* scales, int M, uint64_t d,
+                           const float* ref, int norm, float quot_eps, int codec, uint64_t B,
+                           int s, float* out) {
+    tngo_decode_aggregate2(codes, scales, M, d, ref, NULL, norm, quot_eps, codec, B, s, out);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -460,6 +489,7 @@ struct tngo_state {
     int head;   /* slot of the newest vector */
     uint32_t t; /* rounds done */
     float* ref;
+    float* ref2; /* second reference (combined form) */
     uint32_t* codes;
     float* scales;
     double gram[TNGO_MAX_K * TNGO_MAX_K + TNGO_MAX_K + 1];
@@ -471,13 +501,14 @@ struct tngo_state {
 tngo_state* tngo_create(uint64_t d, int M, int K, int codec, int norm) {
     if (d == 0 || M < 1 || M > 64 || K < 1 || K > TNGO_MAX_K) return NULL;
     if (codec != 1 && codec != 2 && codec != 4) return NULL;
-    if (norm < 0 || norm > 2) return NULL;
+    if (norm < 0 || norm > 3) return NULL;
     tngo_state* st = (tngo_state*)calloc(1, sizeof *st);
     st->d = d; st->M = M; st->K = K; st->codec = codec; st->norm = norm;
     st->B = 128; st->s = 7; st->scale_kind = TNGO_SCALE_ABSMAX; st->fuse_mode = 0;
     st->seed_lo = 0; st->seed_hi = 0; st->ridge = 1e-6; st->quot_eps = 0x1p-4f; st->ref_every = 1;
     st->H = (float*)calloc((size_t)K * d, sizeof(float));
     st->ref = (float*)calloc(d, sizeof(float));
+    st->ref2 = (float*)calloc(d, sizeof(float));
     st->codes = (uint32_t*)calloc((size_t)M * tngo_words_per_worker(d, codec), sizeof(uint32_t));
     st->scales = NULL;
     st->k = 0; st->head = K - 1; st->t = 0;
@@ -486,7 +517,7 @@ tngo_state* tngo_create(uint64_t d, int M, int K, int codec, int norm) {
 
 void tngo_destroy(tngo_state* st) {
     if (!st) return;
-    free(st->H); free(st->ref); free(st->codes); free(st->scales);
+    free(st->H); free(st->ref); free(st->ref2); free(st->codes); free(st->scales);
     free(st);
 }
 
@@ -545,10 +576,12 @@ void tngo_stage_fuse(tngo_state* st, const float* grads, uint64_t ld) {
     memset(st->alpha64, 0, sizeof st->alpha64);
     if (k == 0) { /* empty trajectory: reference = zeros (Algorithm 1 initialisation) */
         memset(st->ref, 0, sizeof(float) * st->d);
+        memset(st->ref2, 0, sizeof(float) * st->d);
         return;
     }
     const float* h[TNGO_MAX_K];
     for (int j = 0; j < k; ++j) h[j] = tngo_history(st, j);
+    if (st->norm == TNGO_NORM_COMB) tngo_magnitude_reference(h, k, st->d, st->ref2);
     int mode = effective_fuse_mode(st);
     if (mode == TNGO_FUSE_LAST) {
         st->alpha[0] = 1.0f; st->alpha64[0] = 1.0;
@@ -566,13 +599,13 @@ void tngo_stage_fuse(tngo_state* st, const float* grads, uint64_t ld) {
 void tngo_stage_encode(tngo_state* st, const float* grads, uint64_t ld) {
     uint64_t nblk = tngo_num_blocks(st->d, st->B);
     if (!st->scales) st->scales = (float*)calloc((size_t)st->M * nblk, sizeof(float));
-    tngo_encode(grads, st->M, ld, st->d, st->ref, st->norm, st->quot_eps, st->codec, st->B, st->s,
-                st->scale_kind, st->seed_lo, st->seed_hi, st->t, st->codes, st->scales);
+    tngo_encode_at(grads, st->M, ld, st->d, st->ref, st->ref2, st->norm, st->quot_eps, st->codec, st->B, st->s,
+                   st->scale_kind, st->seed_lo, st->seed_hi, st->t, 0, st->codes, st->scales);
 }
 
 void tngo_stage_decode_push(tngo_state* st, float* out) {
-    tngo_decode_aggregate(st->codes, st->scales, st->M, st->d, st->ref, st->norm, st->quot_eps,
-                          st->codec, st->B, st->s, out);
+    tngo_decode_aggregate2(st->codes, st->scales, st->M, st->d, st->ref, st->ref2, st->norm, st->quot_eps,
+                           st->codec, st->B, st->s, out);
     push(st, out);
     st->t += 1;
 }
@@ -586,6 +619,7 @@ void tngo_step(tngo_state* st, const float* grads, uint64_t ld, float* out) {
 }
 
 const float* tngo_ref(const tngo_state* st) { return st->ref; }
+const float* tngo_ref2(const tngo_state* st) { return st->ref2; }
 const uint32_t* tngo_codes(const tngo_state* st) { return st->codes; }
 const float* tngo_scales(const tngo_state* st) { return st->scales; }
 const float* tngo_alpha(const tngo_state* st) { return st->alpha; }

@@ -29,7 +29,7 @@ extern "C" {
 
 /* codec value = bits per symbol */
 enum { TNGO_CODEC_SIGN1 = 1, TNGO_CODEC_TERN2 = 2, TNGO_CODEC_QSGD4 = 4 };
-enum { TNGO_NORM_NONE = 0, TNGO_NORM_DIFF = 1, TNGO_NORM_QUOT = 2 };
+enum { TNGO_NORM_NONE = 0, TNGO_NORM_DIFF = 1, TNGO_NORM_QUOT = 2, TNGO_NORM_COMB = 3 };
 enum { TNGO_SCALE_ABSMAX = 0, TNGO_SCALE_L2 = 1 };
 enum { TNGO_FUSE_LAST = 1, TNGO_FUSE_MEAN = 2, TNGO_FUSE_LSQ = 3, TNGO_FUSE_HINDSIGHT = 4 };
 
@@ -81,14 +81,21 @@ void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float
 
 /* Same for a window of a longer vector: the d coordinates are i0 .. i0+d-1 of it (i0 a
  * multiple of 128 and of B), which only moves the Philox counters. */
-void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
-                    float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
+/* ref2: second reference of the combined form r = Q[(g - ref) ./ ref2], v = ref2 . r + ref
+ * (Section 3, display after Eq. 3); only read when norm == TNGO_NORM_COMB. */
+void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, const float* ref2,
+                    int norm, float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
                     uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales);
+/* r'_d = (1/k) sum_j |h_j,d|: per-coordinate magnitude of the trajectory (fp32 fma chain). */
+void tngo_magnitude_reference(const float* const* h, int k, uint64_t d, float* ref2);
 
 /* ---- decode + aggregate + de-normalise (Eq. 2 / Eq. 3, Algorithm 1 "average") */
 void tngo_decode_aggregate(const uint32_t* codes, const float* scales, int M, uint64_t d,
                            const float* ref, int norm, float quot_eps, int codec, uint64_t B,
                            int s, float* out);
+void tngo_decode_aggregate2(const uint32_t* codes, const float* scales, int M, uint64_t d,
+                            const float* ref, const float* ref2, int norm, float quot_eps, int codec,
+                            uint64_t B, int s, float* out);
 /* Decoded value of one symbol (used by tests that unpack the wire themselves). */
 float tngo_dequant(int codec, int s, uint32_t symbol, float R);
 
@@ -113,6 +120,7 @@ void tngo_stage_encode(tngo_state* st, const float* grads, uint64_t ld);
 void tngo_stage_decode_push(tngo_state* st, float* out);
 /* Borrowed views of the state. */
 const float* tngo_ref(const tngo_state* st);
+const float* tngo_ref2(const tngo_state* st);
 const uint32_t* tngo_codes(const tngo_state* st);
 const float* tngo_scales(const tngo_state* st);
 const float* tngo_alpha(const tngo_state* st);

@@ -431,3 +431,76 @@ def test_encoding_a_window_equals_the_window_of_the_whole_encode(codec):
         # and without the offset the random draws differ
         wc0, _ = oracle.encode(np.ascontiguousarray(g[:, i0:i0 + n]), r[i0:i0 + n], norm, codec, B=128, s=5, seed=(7, 1), t=3)
         assert not np.array_equal(wc0, wc)
+
+
+# ---- combined form of Section 3: r = Q[(g - ref) ./ ref2], v = ref2 . r + ref -------------------
+def _comb_inputs(seed=9, d=128 * 6 + 30, M=4):
+    rng = np.random.default_rng(seed)
+    g = rng.standard_normal((M, d)).astype(np.float32)
+    r = (0.7 * g.mean(0) + 0.2 * rng.standard_normal(d)).astype(np.float32)
+    r2 = np.abs(rng.standard_normal(d)).astype(np.float32) + 0.25
+    return g, r, r2
+
+
+def test_combined_form_with_unit_second_reference_is_the_difference_form():
+    g, r, _ = _comb_inputs()
+    ones = np.ones_like(r)
+    for codec in (oracle.CODEC_SIGN1, oracle.CODEC_TERN2, oracle.CODEC_QSGD4):
+        a = oracle.encode(g, r, oracle.NORM_COMB, codec, seed=(3, 0), t=2, ref2=ones)
+        b = oracle.encode(g, r, oracle.NORM_DIFF, codec, seed=(3, 0), t=2)
+        assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+        oa = oracle.decode_aggregate(a[0], a[1], g.shape[1], r, oracle.NORM_COMB, codec, ref2=ones)
+        ob = oracle.decode_aggregate(b[0], b[1], g.shape[1], r, oracle.NORM_DIFF, codec)
+        assert np.array_equal(oa, ob)
+
+
+def test_combined_form_with_zero_first_reference_is_the_quotient_form():
+    g, _, r2 = _comb_inputs()
+    zeros = np.zeros_like(r2)
+    a = oracle.encode(g, zeros, oracle.NORM_COMB, oracle.CODEC_TERN2, seed=(3, 0), t=2, ref2=r2)
+    b = oracle.encode(g, r2, oracle.NORM_QUOT, oracle.CODEC_TERN2, seed=(3, 0), t=2)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1], b[1])
+    oa = oracle.decode_aggregate(a[0], a[1], g.shape[1], zeros, oracle.NORM_COMB, oracle.CODEC_TERN2, ref2=r2)
+    ob = oracle.decode_aggregate(b[0], b[1], g.shape[1], r2, oracle.NORM_QUOT, oracle.CODEC_TERN2)
+    assert np.array_equal(oa, ob)
+
+
+def test_combined_form_gradient_equal_to_reference_gives_zero_codes_and_returns_it():
+    _, r, r2 = _comb_inputs()
+    g = np.repeat(r[None], 3, axis=0)
+    codes, scales = oracle.encode(g, r, oracle.NORM_COMB, oracle.CODEC_TERN2, ref2=r2)
+    assert not codes.any() and not scales.any()
+    out = oracle.decode_aggregate(codes, scales, r.shape[0], r, oracle.NORM_COMB, oracle.CODEC_TERN2, ref2=r2)
+    assert np.array_equal(out, r)
+
+
+def test_combined_form_is_unbiased_and_scales_blocks_by_the_second_reference():
+    g, r, r2 = _comb_inputs(d=256, M=1)
+    S = 4000
+    acc = np.zeros(g.shape[1])
+    for t in range(S):
+        c, sc = oracle.encode(g, r, oracle.NORM_COMB, oracle.CODEC_TERN2, seed=(1, 2), t=t, ref2=r2)
+        acc += oracle.decode_aggregate(c, sc, g.shape[1], r, oracle.NORM_COMB, oracle.CODEC_TERN2, ref2=r2)
+    mean = acc / S
+    den = oracle.quot_den(r2)
+    v = (g[0] - r) / den
+    R = np.repeat(np.abs(v).reshape(-1, 128).max(1), 128)
+    sigma = den * np.sqrt(np.maximum(R * np.abs(v) - v * v, 0) / S)     # closed-form variance of the ternary code, rescaled
+    assert np.all(np.abs(mean - g[0]) <= 5 * sigma + 1e-5)
+    # the scale on the wire is max |(g - ref) / den| over the block
+    _, sc = oracle.encode(g, r, oracle.NORM_COMB, oracle.CODEC_TERN2, ref2=r2)
+    assert np.allclose(sc[0], np.abs(v).reshape(-1, 128).max(1), rtol=1e-6)
+
+
+def test_magnitude_reference_is_the_mean_absolute_value_of_the_history():
+    rng = np.random.default_rng(4)
+    hist = [rng.standard_normal(500).astype(np.float32) for _ in range(5)]
+    got = oracle.magnitude_reference(hist)
+    want = np.mean(np.abs(np.stack(hist).astype(np.float64)), axis=0)
+    assert np.allclose(got, want, rtol=1e-6)
+    assert np.array_equal(oracle.magnitude_reference([hist[0]]), np.abs(hist[0]))   # k = 1: exactly |h_1|
+    st = oracle.State(500, 2, 5, oracle.CODEC_TERN2, oracle.NORM_COMB, fuse_mode=oracle.FUSE_MEAN)
+    for h in hist[::-1]:
+        st.push_reference(h)
+    st.fuse(rng.standard_normal((2, 500)).astype(np.float32))
+    assert np.array_equal(st.ref2(), got)
