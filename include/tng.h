@@ -48,7 +48,10 @@ typedef enum {
 
 /* value = bits per coordinate symbol */
 typedef enum { TNG_CODEC_SIGN1 = 1, TNG_CODEC_TERN2 = 2, TNG_CODEC_QSGD4 = 4 } tng_codec;
-typedef enum { TNG_NORM_NONE = 0, TNG_NORM_DIFF = 1, TNG_NORM_QUOT = 2 } tng_norm_mode;
+/* NONE: v = g.  DIFF: Eq. 2.  QUOT: Eq. 3.  COMB: the combined form of Section 3,
+ * r = Q[(g - ref) ./ ref'], v = ref' . r + ref, with ref' = the mean absolute value of the
+ * stored aggregates (per coordinate), guarded like the quotient form's denominator. */
+typedef enum { TNG_NORM_NONE = 0, TNG_NORM_DIFF = 1, TNG_NORM_QUOT = 2, TNG_NORM_COMB = 3 } tng_norm_mode;
 typedef enum {
     TNG_FUSE_AUTO = 0,     /* K == 1 -> LAST, else LSQ */
     TNG_FUSE_LAST = 1,     /* r = newest aggregate (delayed gradient, Sec. 3.1 / Sec. 4.2 protocol) */

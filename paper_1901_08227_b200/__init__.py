@@ -9,4 +9,4 @@ library, or a round without a CUDA device, raises.
 from . import tng  # noqa: F401
 from .tng import (  # noqa: F401
     CODEC_QSGD4, CODEC_SIGN1, CODEC_TERN2, FUSE_AUTO, FUSE_HINDSIGHT, FUSE_LAST, FUSE_LSQ, FUSE_MEAN, NORM_DIFF,
-    NORM_NONE, NORM_QUOT, SCALE_ABSMAX, SCALE_L2, Context, TngError)
+    NORM_COMB, NORM_NONE, NORM_QUOT, SCALE_ABSMAX, SCALE_L2, Context, TngError)

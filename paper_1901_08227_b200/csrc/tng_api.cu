@@ -40,7 +40,7 @@ struct tng_ctx {
     size_t ws_bytes = 0;
     bool ws_owned = false, ws_ready = false;
     size_t off_ring = 0, off_ref = 0, off_codes = 0, off_scales = 0, off_tile_stat = 0, off_tree = 0,
-           off_partials = 0, off_fb = 0, off_stage_g = 0, off_stage_o = 0;
+           off_partials = 0, off_fb = 0, off_stage_g = 0, off_stage_o = 0, off_ref2 = 0;
     // state
     uint32_t k = 0;
     int head = 0;
@@ -49,6 +49,7 @@ struct tng_ctx {
     int last_mode = TNG_FUSE_LAST;
     bool last_had_stats = false;
     bool last_solved = false;         // the last fusion ran the solve kernel (alpha lives on the device)
+    bool ref2_valid = false;          // combined form: the second-reference buffer has been written
     // bookkeeping
     int device = 0, sm_count = 148;
     cudaStream_t last_stream = nullptr;
@@ -65,6 +66,7 @@ struct tng_ctx {
 
     float* ring(int slot) const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_ring) + (size_t)slot * d_pad; }
     float* ref_buf() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_ref); }
+    float* ref2_buf() const { return norm == TNG_NORM_COMB ? reinterpret_cast<float*>(static_cast<char*>(ws) + off_ref2) : nullptr; }
     uint32_t* codes() const { return reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + off_codes); }
     float* scales() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_scales); }
     float* tile_stat() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_tile_stat); }
@@ -109,6 +111,7 @@ void size_ctx(tng_ctx* c) {
     size_t off = 0;
     c->off_ring = off;      off += align_up((size_t)c->K * c->d_pad * sizeof(float));
     c->off_ref = off;       off += align_up((size_t)c->d_pad * sizeof(float));
+    c->off_ref2 = off;      off += align_up(c->norm == TNG_NORM_COMB ? (size_t)c->d_pad * sizeof(float) : 0);
     c->off_codes = off;     off += align_up((size_t)c->M * g.wpw * sizeof(uint32_t));
     c->off_scales = off;    off += align_up((size_t)c->M * g.nblk * sizeof(float));
     const bool general = g.block != TNG_TILE;
@@ -202,13 +205,17 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
     int launches = 0;
     if (c->k == 0) {   // empty trajectory: reference = zeros (initial state of Algorithm 1)
         TNG_CUDA(c, cudaMemsetAsync(c->ref_buf(), 0, c->d_pad * sizeof(float), st));
+        if (c->ref2_buf()) {
+            TNG_CUDA(c, cudaMemsetAsync(c->ref2_buf(), 0, c->d_pad * sizeof(float), st));
+            c->ref2_valid = true;
+        }
         c->ref_cur = c->ref_buf();
         if (tm) { tm->mark(0, false); tm->mark(1, false); tm->mark(2, false); }
         return TNG_OK;
     }
     const float* rows[kMaxK];
     for (uint32_t j = 0; j < c->k; ++j) rows[j] = c->ring(c->hist_slot(j));
-    if (mode == TNG_FUSE_LAST) {   // delayed-gradient reference: alias the newest slot, no pass
+    if (mode == TNG_FUSE_LAST && c->norm != TNG_NORM_COMB) {   // delayed-gradient reference: alias the newest slot, no pass
         c->ref_cur = rows[0];
         if (tm) { tm->mark(0, false); tm->mark(1, false); tm->mark(2, false); }
         return TNG_OK;
@@ -228,12 +235,14 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
         defer->k = (int)c->k;
         defer->alpha = c->fb()->alpha32;
         defer->ref_out = c->ref_buf();
+        defer->ref2_out = c->ref2_buf();
         if (tm) tm->mark(2, false);
     } else {
-        TNG_CUDA(c, launch_combine(rows, (int)c->k, c->d, c->fb(), c->ref_buf(), c->sm_count, st, &launches));
+        TNG_CUDA(c, launch_combine(rows, (int)c->k, c->d, c->fb(), c->ref_buf(), c->ref2_buf(), c->sm_count, st, &launches));
         if (tm) tm->mark(2, true);
     }
     c->ref_cur = c->ref_buf();
+    if (c->ref2_buf()) c->ref2_valid = true;
     c->launches += (uint64_t)launches;
     return TNG_OK;
 }
@@ -241,7 +250,7 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
 tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* ref, const RefFusion* fusion, uint32_t step,
                      cudaStream_t st) {
     int launches = 0;
-    TNG_CUDA(c, launch_encode(c->geom, grads, ld, ref, fusion, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
+    TNG_CUDA(c, launch_encode(c->geom, grads, ld, ref, c->ref2_buf(), fusion, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
                               c->fb(), c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
@@ -249,7 +258,7 @@ tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* r
 
 tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, cudaStream_t st) {
     int launches = 0;
-    TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), ref, out_a, out_b, c->fb(), c->sm_count, st, &launches));
+    TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), ref, c->ref2_buf(), out_a, out_b, c->fb(), c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
 }
@@ -294,7 +303,7 @@ tng_status tng_create(tng_ctx** out, uint64_t d, uint32_t M, uint32_t K, tng_cod
     *out = nullptr;
     if (d < 1 || d > TNG_MAX_COORDS || M < 1 || M > TNG_MAX_WORKERS || K < 1 || K > TNG_MAX_HISTORY) return TNG_ERR_INVALID_ARG;
     if (codec != TNG_CODEC_SIGN1 && codec != TNG_CODEC_TERN2 && codec != TNG_CODEC_QSGD4) return TNG_ERR_INVALID_ARG;
-    if (norm != TNG_NORM_NONE && norm != TNG_NORM_DIFF && norm != TNG_NORM_QUOT) return TNG_ERR_INVALID_ARG;
+    if (norm != TNG_NORM_NONE && norm != TNG_NORM_DIFF && norm != TNG_NORM_QUOT && norm != TNG_NORM_COMB) return TNG_ERR_INVALID_ARG;
     tng_ctx* c = new (std::nothrow) tng_ctx();
     if (!c) return TNG_ERR_ALLOC;
     c->d = d; c->M = M; c->K = K; c->codec = (int)codec; c->norm = (int)norm;
@@ -436,7 +445,7 @@ void fill_header(const tng_ctx* c, StateHeader* h) {
 
 tng_status tng_state_bytes(tng_ctx* c, size_t* bytes) {
     if (!c || !bytes) return TNG_ERR_INVALID_ARG;
-    *bytes = sizeof(StateHeader) + ((size_t)c->K + 1) * c->d * sizeof(float);
+    *bytes = sizeof(StateHeader) + ((size_t)c->K + 2) * c->d * sizeof(float);
     return TNG_OK;
 }
 
@@ -448,6 +457,7 @@ tng_status tng_save_state(tng_ctx* c, void* host_buf, size_t bytes, size_t* writ
     StateHeader h;
     fill_header(c, &h);
     h.has_ref = (c->ref_every > 1 && c->ref_cur) ? 1u : 0u;
+    if (h.has_ref && c->norm == TNG_NORM_COMB) h.has_ref = c->ref2_valid ? 2u : 0u;   // both references or none
     const size_t vec = c->d * sizeof(float);
     const size_t need = sizeof h + ((size_t)c->k + h.has_ref) * vec;
     if (bytes < need) return TNG_ERR_ALLOC;
@@ -457,6 +467,7 @@ tng_status tng_save_state(tng_ctx* c, void* host_buf, size_t bytes, size_t* writ
     for (uint32_t j = 0; j < c->k; ++j, p += vec)   // newest first
         TNG_CUDA(c, cudaMemcpyAsync(p, c->ring(c->hist_slot(j)), vec, cudaMemcpyDeviceToHost, st));
     if (h.has_ref) TNG_CUDA(c, cudaMemcpyAsync(p, c->ref_cur, vec, cudaMemcpyDeviceToHost, st));
+    if (h.has_ref == 2) TNG_CUDA(c, cudaMemcpyAsync(p + vec, c->ref2_buf(), vec, cudaMemcpyDeviceToHost, st));
     TNG_CUDA(c, cudaStreamSynchronize(st));
     if (written) *written = need;
     return TNG_OK;
@@ -470,7 +481,8 @@ tng_status tng_load_state(tng_ctx* c, const void* host_buf, size_t bytes, void* 
     if (h.magic != kStateMagic || h.version != 1 || h.d != mine.d || h.M != mine.M || h.K != mine.K || h.codec != mine.codec ||
         h.norm != mine.norm || h.block != mine.block || h.levels != mine.levels || h.scale_kind != mine.scale_kind ||
         h.fuse_mode != mine.fuse_mode || h.seed_lo != mine.seed_lo || h.seed_hi != mine.seed_hi || h.ref_every != mine.ref_every ||
-        h.ridge != mine.ridge || h.quot_eps != mine.quot_eps || h.k > h.K || h.has_ref > 1)
+        h.ridge != mine.ridge || h.quot_eps != mine.quot_eps || h.k > h.K || h.has_ref > 2 ||
+        (h.has_ref == 2) != (h.has_ref != 0 && c->norm == TNG_NORM_COMB))
         return TNG_ERR_INVALID_ARG;
     const size_t vec = c->d * sizeof(float);
     if (bytes < sizeof h + ((size_t)h.k + h.has_ref) * vec) return TNG_ERR_INVALID_ARG;
@@ -482,7 +494,9 @@ tng_status tng_load_state(tng_ctx* c, const void* host_buf, size_t bytes, void* 
     for (uint32_t j = 0; j < h.k; ++j, p += vec)
         TNG_CUDA(c, cudaMemcpyAsync(c->ring((int)(h.k - 1 - j)), p, vec, cudaMemcpyHostToDevice, st));
     if (h.has_ref) TNG_CUDA(c, cudaMemcpyAsync(c->ref_buf(), p, vec, cudaMemcpyHostToDevice, st));
+    if (h.has_ref == 2) TNG_CUDA(c, cudaMemcpyAsync(c->ref2_buf(), p + vec, vec, cudaMemcpyHostToDevice, st));
     TNG_CUDA(c, cudaStreamSynchronize(st));
+    c->ref2_valid = h.has_ref == 2;
     c->k = h.k;
     c->head = h.k ? (int)h.k - 1 : 0;
     c->rounds = h.rounds;
@@ -513,6 +527,7 @@ tng_status tng_encode(tng_ctx* c, const float* grads_dev, uint64_t ld, const flo
     if (s != TNG_OK) return s;
     const float* ref = ref_dev ? ref_dev : c->ref_cur;
     if (!ref && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;   // no fusion has produced a reference yet
+    if (c->norm == TNG_NORM_COMB && !c->ref2_valid) return TNG_ERR_STATE;   // the second reference comes from a fusion
     return do_encode(c, grads_dev, ld, ref, nullptr, step, st);
 }
 
@@ -524,6 +539,7 @@ tng_status tng_decode_aggregate(tng_ctx* c, const float* ref_dev, float* out_dev
     if (s != TNG_OK) return s;
     const float* ref = ref_dev ? ref_dev : c->ref_cur;
     if (!ref && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;
+    if (c->norm == TNG_NORM_COMB && !c->ref2_valid) return TNG_ERR_STATE;
     return do_decode(c, ref, out_dev, nullptr, st);
 }
 

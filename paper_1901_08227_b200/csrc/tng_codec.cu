@@ -45,6 +45,11 @@ struct EncodeArgs {
     const float* alpha;
     float* ref_out;
     int hist_k;
+    // combined form (TNG_NORM_COMB): second reference r' = (1/k) sum_j |h_j|, read from ref2 or,
+    // when the reference is combined here, formed alongside it (weight inv_k) and written to ref2_out
+    const float* ref2;
+    float* ref2_out;
+    float inv_k;
 };
 
 // max(|a|, |b|) that returns NaN if either is NaN
@@ -63,8 +68,41 @@ __device__ __forceinline__ float absmax_nan2(float a, float b) {
 // ballots), so work that can run on the multiplier pipe is put there: addresses are
 // 32 x 32 -> 64 multiply-adds and the uniform's shift is a high multiply.
 // v = g - r (Eq. 2), v = g * (1/den) (Eq. 3), or v = g
+// operands of the normalisation for the lane's four coordinates: a = r (difference and combined
+// forms) or 1/den (quotient form); b = 1/den' (combined form only)
+struct NormOp {
+    float4 a, b;
+};
+
+// the reference(s) of a tile -> normalisation operands
 template <int NORM>
-__device__ __forceinline__ void encode_normalise(const float4 g, const float4 op, float (&v)[4]) {
+__device__ __forceinline__ NormOp make_norm_op(const float4 r, const float4 r2, const float quot_eps) {
+    NormOp op;
+    op.a = make_float4(0.f, 0.f, 0.f, 0.f);
+    op.b = op.a;
+    if (NORM == TNG_NORM_DIFF || NORM == TNG_NORM_COMB) op.a = r;
+    if (NORM == TNG_NORM_QUOT || NORM == TNG_NORM_COMB) {
+        const float4 den = quot_den4(NORM == TNG_NORM_QUOT ? r : r2, quot_eps);
+        const float4 inv = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z), __fdiv_rn(1.0f, den.w));
+        if (NORM == TNG_NORM_QUOT) op.a = inv; else op.b = inv;
+    }
+    return op;
+}
+
+// r' += inv_k * |h| (the second reference's fma chain)
+__device__ __forceinline__ void magnitude_fma(float4& r2, const float inv_k, const float4 h) {
+    r2.x = __fmaf_rn(inv_k, fabsf(h.x), r2.x); r2.y = __fmaf_rn(inv_k, fabsf(h.y), r2.y);
+    r2.z = __fmaf_rn(inv_k, fabsf(h.z), r2.z); r2.w = __fmaf_rn(inv_k, fabsf(h.w), r2.w);
+}
+
+template <int NORM>
+__device__ __forceinline__ void encode_normalise(const float4 g, const NormOp& opn, float (&v)[4]) {
+    const float4 op = opn.a;
+    if (NORM == TNG_NORM_COMB) {   // v = (g - r) * (1/den'), two roundings
+        v[0] = __fmul_rn(__fsub_rn(g.x, op.x), opn.b.x); v[1] = __fmul_rn(__fsub_rn(g.y, op.y), opn.b.y);
+        v[2] = __fmul_rn(__fsub_rn(g.z, op.z), opn.b.z); v[3] = __fmul_rn(__fsub_rn(g.w, op.w), opn.b.w);
+        return;
+    }
     if (NORM == TNG_NORM_DIFF) {
         v[0] = __fsub_rn(g.x, op.x); v[1] = __fsub_rn(g.y, op.y); v[2] = __fsub_rn(g.z, op.z); v[3] = __fsub_rn(g.w, op.w);
     } else if (NORM == TNG_NORM_QUOT) {
@@ -124,7 +162,7 @@ __device__ __forceinline__ void encode_quantise(const EncodeArgs& a, const float
 }
 
 template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL>
-__device__ __forceinline__ bool encode_symbols(const EncodeArgs& a, const float4 g, const float4 op,
+__device__ __forceinline__ bool encode_symbols(const EncodeArgs& a, const float4 g, const NormOp& op,
                                                const uint32_t m, const uint64_t T, const uint4 x, const uint64_t blk,
                                                const int lane, const uint32_t valid, uint32_t (&w)[4 * CODEC], float& R) {
     float v[4];
@@ -146,7 +184,7 @@ __device__ __forceinline__ bool encode_symbols(const EncodeArgs& a, const float4
 
 // encode_symbols, then lane 0 writes the words every lane holds (and the scale)
 template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL>
-__device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const float4 g, const float4 op,
+__device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const float4 g, const NormOp& op,
                                                   const uint32_t m, const uint64_t T, const uint32_t q_lo,
                                                   const uint32_t q_hi, const uint64_t blk, const int lane,
                                                   const uint32_t valid) {
@@ -185,9 +223,9 @@ __device__ __forceinline__ void encode_tile(const EncodeArgs& a, const float* s_
     for (int k = 0; k < kWorkerBatch; ++k)
         if ((uint32_t)k < a.M) g[k] = load_row(k);
 
-    float4 op = make_float4(0.f, 0.f, 0.f, 0.f);
+    NormOp op = make_norm_op<TNG_NORM_NONE>(make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f), 0.f);
     if (NORM != TNG_NORM_NONE) {
-        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
         if (FUSEREF) {
             for (int j0 = 0; j0 < a.hist_k; j0 += 4) {
                 float4 h[4];
@@ -201,20 +239,20 @@ __device__ __forceinline__ void encode_tile(const EncodeArgs& a, const float* s_
                         const float al = s_alpha[j0 + jj];
                         r.x = __fmaf_rn(al, h[jj].x, r.x); r.y = __fmaf_rn(al, h[jj].y, r.y);
                         r.z = __fmaf_rn(al, h[jj].z, r.z); r.w = __fmaf_rn(al, h[jj].w, r.w);
+                        if (NORM == TNG_NORM_COMB) magnitude_fma(r2, a.inv_k, h[jj]);
                     }
             }
             if (FULL) *reinterpret_cast<float4*>(a.ref_out + i0) = r;
             else store4(a.ref_out, i0, a.d, r);
-        } else if (a.ref) {
-            r = FULL ? *reinterpret_cast<const float4*>(a.ref + i0) : load4(a.ref, i0, a.d);
-        }
-        if (NORM == TNG_NORM_DIFF) {
-            op = r;
+            if (NORM == TNG_NORM_COMB) {
+                if (FULL) *reinterpret_cast<float4*>(a.ref2_out + i0) = r2;
+                else store4(a.ref2_out, i0, a.d, r2);
+            }
         } else {
-            const float4 den = quot_den4(r, a.quot_eps);
-            op = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z),
-                             __fdiv_rn(1.0f, den.w));
+            if (a.ref) r = FULL ? *reinterpret_cast<const float4*>(a.ref + i0) : load4(a.ref, i0, a.d);
+            if (NORM == TNG_NORM_COMB && a.ref2) r2 = FULL ? *reinterpret_cast<const float4*>(a.ref2 + i0) : load4(a.ref2, i0, a.d);
         }
+        op = make_norm_op<NORM>(r, r2, a.quot_eps);
     }
     const uint64_t blk = (PHASE == kPhaseQuant) ? (T * kTile) / a.block : T;
     const uint64_t q = T * 32u + (uint32_t)lane;                 // Philox counter of the lane's four coordinates
@@ -322,8 +360,8 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
         const uint64_t T = c * kEncPipeWarps + (uint32_t)warp;
         const uint64_t q = T * 32u + (uint32_t)lane;
         const uint32_t q_lo = (uint32_t)q, q_hi = (uint32_t)(q >> 32);
-        // ---- the reference of the tile
-        float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+        // ---- the reference(s) of the tile
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
         for (int p0 = 0; p0 < n_pre; p0 += G::kRows) {
             const int n = (n_pre - p0 < G::kRows) ? n_pre - p0 : G::kRows;
             const uint32_t s = it % G::kStages, use = it / G::kStages;
@@ -338,25 +376,21 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                     const float al = s_alpha[p0 + j];
                     r.x = __fmaf_rn(al, x.x, r.x); r.y = __fmaf_rn(al, x.y, r.y);
                     r.z = __fmaf_rn(al, x.z, r.z); r.w = __fmaf_rn(al, x.w, r.w);
+                    if (NORM == TNG_NORM_COMB) magnitude_fma(r2, a.inv_k, x);
                 }
-            } else {
+            } else {   // the reference itself, then (combined form) the second reference
                 r = *reinterpret_cast<const float4*>(base);
+                if (NORM == TNG_NORM_COMB && n > 1) r2 = *reinterpret_cast<const float4*>(base + G::kRowBytes);
             }
             __syncwarp();
             if (lane == 0) mbar_arrive(pipe.empty(s));
             ++it;
         }
-        float4 op = make_float4(0.f, 0.f, 0.f, 0.f);
-        if (NORM != TNG_NORM_NONE) {
-            if (FUSEREF) *reinterpret_cast<float4*>(a.ref_out + (T * kTile + (uint64_t)lane * 4u)) = r;
-            if (NORM == TNG_NORM_DIFF) {
-                op = r;
-            } else {
-                const float4 den = quot_den4(r, a.quot_eps);
-                op = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z),
-                                 __fdiv_rn(1.0f, den.w));
-            }
+        if (FUSEREF) {
+            *reinterpret_cast<float4*>(a.ref_out + (T * kTile + (uint64_t)lane * 4u)) = r;
+            if (NORM == TNG_NORM_COMB) *reinterpret_cast<float4*>(a.ref2_out + (T * kTile + (uint64_t)lane * 4u)) = r2;
         }
+        const NormOp op = make_norm_op<NORM>(r, r2, a.quot_eps);
         // ---- the gradient rows, one fill of up to 8 workers at a time.  Every lane ends up with
         // all words of every worker; lane k writes worker k of the fill through a pointer it
         // computes once per fill, and the fill's scales go out as one store.
@@ -471,6 +505,7 @@ struct DecodeArgs {
     const uint32_t* codes;
     const float* scales;
     const float* ref;
+    const float* ref2;     // second reference (combined form)
     float* out_a;
     float* out_b;
     uint32_t* pipe_error;
@@ -536,7 +571,8 @@ __device__ __forceinline__ void decode_worker(const uint32_t (&w)[4 * CODEC], co
 
 // average over the M workers (Algorithm 1), put the reference back (Eq. 2 / Eq. 3), store
 template <int NORM, bool FULL>
-__device__ __forceinline__ void decode_finish(const DecodeArgs& a, const float (&acc)[4], const float4 r, const uint64_t i0) {
+__device__ __forceinline__ void decode_finish(const DecodeArgs& a, const float (&acc)[4], const float4 r, const float4 r2,
+                                              const uint64_t i0) {
     float4 o;
     if (a.inv_m > 0.0f) {
         o.x = __fmul_rn(acc[0], a.inv_m); o.y = __fmul_rn(acc[1], a.inv_m); o.z = __fmul_rn(acc[2], a.inv_m); o.w = __fmul_rn(acc[3], a.inv_m);
@@ -549,6 +585,10 @@ __device__ __forceinline__ void decode_finish(const DecodeArgs& a, const float (
     } else if (NORM == TNG_NORM_QUOT) {
         const float4 den = quot_den4(r, a.quot_eps);
         o.x = __fmul_rn(den.x, o.x); o.y = __fmul_rn(den.y, o.y); o.z = __fmul_rn(den.z, o.z); o.w = __fmul_rn(den.w, o.w);
+    } else if (NORM == TNG_NORM_COMB) {   // out = den' * a + r, two roundings
+        const float4 den = quot_den4(r2, a.quot_eps);
+        o.x = __fadd_rn(__fmul_rn(den.x, o.x), r.x); o.y = __fadd_rn(__fmul_rn(den.y, o.y), r.y);
+        o.z = __fadd_rn(__fmul_rn(den.z, o.z), r.z); o.w = __fadd_rn(__fmul_rn(den.w, o.w), r.w);
     }
     if (FULL) {
         if (a.out_a) *reinterpret_cast<float4*>(a.out_a + i0) = o;
@@ -636,20 +676,23 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
     uint64_t T = a.tile_begin + gwarp;
     uint4 cw = make_uint4(0u, 0u, 0u, 0u);
     float sc = 0.0f;
-    float4 r = make_float4(0.f, 0.f, 0.f, 0.f);
+    float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
+    const bool has_ref2 = (NORM == TNG_NORM_COMB) && a.ref2 != nullptr;
     if (T < nfull) {
         decode_fetch<CODEC>(a, T, tiled ? T : (T * kTile) / a.block, 0, lane, cw, sc);
         if (has_ref) r = *reinterpret_cast<const float4*>(a.ref + (T * kTile + (uint64_t)lane * 4u));
+        if (has_ref2) r2 = *reinterpret_cast<const float4*>(a.ref2 + (T * kTile + (uint64_t)lane * 4u));
     }
     for (; T < nfull; T += nwarps) {
         slot->cw[lane] = cw;
         slot->sc[lane] = sc;
-        const float4 rcur = r;
+        const float4 rcur = r, r2cur = r2;
         __syncwarp();
         const uint64_t Tn = T + nwarps;
         if (Tn < nfull) {                                            // next tile's loads go out now
             decode_fetch<CODEC>(a, Tn, tiled ? Tn : (Tn * kTile) / a.block, 0, lane, cw, sc);
             if (has_ref) r = *reinterpret_cast<const float4*>(a.ref + (Tn * kTile + (uint64_t)lane * 4u));
+            if (has_ref2) r2 = *reinterpret_cast<const float4*>(a.ref2 + (Tn * kTile + (uint64_t)lane * 4u));
         }
         float acc[4] = {z, z, z, z};
         decode_round<CODEC>(slot, n0, a.levels, pw, lane, acc);
@@ -664,14 +707,15 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
             decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
         }
         __syncwarp();                                                // slot is free again
-        decode_finish<NORM, true>(a, acc, rcur, T * kTile + (uint64_t)lane * 4u);
+        decode_finish<NORM, true>(a, acc, rcur, r2cur, T * kTile + (uint64_t)lane * 4u);
     }
     // the ragged last tile
     if (nfull < a.ntile && gwarp == nfull % nwarps) {
         const uint64_t Tr = nfull, i0 = Tr * kTile + (uint64_t)lane * 4u;
         const uint64_t blk = tiled ? Tr : (Tr * kTile) / a.block;
-        float4 rr = make_float4(0.f, 0.f, 0.f, 0.f);
+        float4 rr = make_float4(0.f, 0.f, 0.f, 0.f), rr2 = rr;
         if (has_ref) rr = load4(a.ref, i0, a.d);
+        if (has_ref2) rr2 = load4(a.ref2, i0, a.d);
         float acc[4] = {z, z, z, z};
         for (uint32_t m0 = 0; m0 < a.M; m0 += kRound) {
             uint4 cw2;
@@ -683,7 +727,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
             __syncwarp();
             decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
         }
-        decode_finish<NORM, false>(a, acc, rr, i0);
+        decode_finish<NORM, false>(a, acc, rr, rr2, i0);
     }
 }
 
@@ -735,6 +779,7 @@ cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t
             for (int j = 0; j < a.hist_k; ++j) pa.rows.row[pa.rows.nrows++] = a.hist[j];
         } else if (NORM != TNG_NORM_NONE && a.ref) {
             pa.rows.row[pa.rows.nrows++] = a.ref;
+            if (NORM == TNG_NORM_COMB && a.ref2) pa.rows.row[pa.rows.nrows++] = a.ref2;
         }
         pa.rows.n_pre = pa.rows.nrows;
         for (uint32_t m = 0; m < a.M; ++m) pa.rows.row[pa.rows.nrows++] = a.grads + (uint64_t)m * a.ld;
@@ -776,6 +821,7 @@ cudaError_t encode_dispatch_norm(const EncodeArgs& a, int norm, int scale, int p
     switch (norm) {
         case TNG_NORM_DIFF: return encode_dispatch_scale<CODEC, TNG_NORM_DIFF>(a, scale, phase, sm_count, st, launches);
         case TNG_NORM_QUOT: return encode_dispatch_scale<CODEC, TNG_NORM_QUOT>(a, scale, phase, sm_count, st, launches);
+        case TNG_NORM_COMB: return encode_dispatch_scale<CODEC, TNG_NORM_COMB>(a, scale, phase, sm_count, st, launches);
         default: return encode_dispatch_scale<CODEC, TNG_NORM_NONE>(a, scale, phase, sm_count, st, launches);
     }
 }
@@ -804,6 +850,7 @@ cudaError_t decode_dispatch_norm(const DecodeArgs& a, int norm, int sm_count, cu
     switch (norm) {
         case TNG_NORM_DIFF: return decode_launch<CODEC, TNG_NORM_DIFF>(a, sm_count, st, launches);
         case TNG_NORM_QUOT: return decode_launch<CODEC, TNG_NORM_QUOT>(a, sm_count, st, launches);
+        case TNG_NORM_COMB: return decode_launch<CODEC, TNG_NORM_COMB>(a, sm_count, st, launches);
         default: return decode_launch<CODEC, TNG_NORM_NONE>(a, sm_count, st, launches);
     }
 }
@@ -820,14 +867,17 @@ size_t tree_tmp_floats(const CodecGeom& g) {
 
 bool encode_can_fuse_reference(const CodecGeom& g) { return g.block == kTile && g.norm != TNG_NORM_NONE; }
 
-cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref, const RefFusion* fusion,
+cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref, const float* ref2,
+                          const RefFusion* fusion,
                           uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp, FuseBlock* fb,
                           int sm_count, cudaStream_t st, int* launches) {
     EncodeArgs a;
     a.hist_k = 0; a.alpha = nullptr; a.ref_out = nullptr;
+    a.ref2 = ref2; a.ref2_out = nullptr; a.inv_k = 0.0f;
     for (int j = 0; j < kMaxK; ++j) a.hist[j] = nullptr;
     if (fusion && fusion->k > 0 && encode_can_fuse_reference(g)) {
         a.hist_k = fusion->k; a.alpha = fusion->alpha; a.ref_out = fusion->ref_out;
+        a.ref2_out = fusion->ref2_out; a.inv_k = 1.0f / (float)fusion->k;
         for (int j = 0; j < fusion->k; ++j) a.hist[j] = fusion->rows[j];
     }
     a.grads = grads; a.ref = ref; a.codes = codes; a.scales = scales; a.tile_stat = tile_stat;
@@ -866,10 +916,10 @@ cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, c
     return encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseQuant, sm_count, st, launches);
 }
 
-cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref,
+cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref, const float* ref2,
                           float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
     DecodeArgs a;
-    a.codes = codes; a.scales = scales; a.ref = ref; a.out_a = out_a; a.out_b = out_b;
+    a.codes = codes; a.scales = scales; a.ref = ref; a.ref2 = ref2; a.out_a = out_a; a.out_b = out_b;
     a.pipe_error = &fb->pipe_error; a.tile_begin = 0;
     a.d = g.d; a.ntile = g.ntile; a.nblk = (uint32_t)g.nblk; a.block = g.block; a.wpw = (uint32_t)g.wpw; a.M = g.M;
     a.one = 1u; a.levels = g.levels; a.quot_eps = g.quot_eps;

@@ -370,6 +370,8 @@ __global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mod
     if (mode == TNG_FUSE_MEAN) {
         const float inv = __fdiv_rn(1.0f, (float)k);
         for (int j = 0; j < k; ++j) alpha[j] = (double)inv;
+    } else if (mode == TNG_FUSE_LAST) {
+        alpha[0] = 1.0;
     } else {
         for (int a = 0; a < k; ++a)   // mirror the upper triangle
             for (int b = 0; b < a; ++b) G[a * kGramStride + b] = G[b * kGramStride + a];
@@ -438,6 +440,8 @@ struct CombineArgs {
     const float* rows[kMaxK];
     const float* alpha;
     float* ref;
+    float* ref2;     // nullptr, or the second reference r' = (1/k) sum_j |h_j|
+    float inv_k;
     uint64_t d;
 };
 
@@ -460,6 +464,15 @@ __global__ void __launch_bounds__(256) combine_kernel(const CombineArgs a) {
             r.z = __fmaf_rn(al[j], h[j].z, r.z); r.w = __fmaf_rn(al[j], h[j].w, r.w);
         }
         store4(a.ref, i0, a.d, r);
+        if (a.ref2) {
+            float4 r2 = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int j = 0; j < KK; ++j) {
+                r2.x = __fmaf_rn(a.inv_k, fabsf(h[j].x), r2.x); r2.y = __fmaf_rn(a.inv_k, fabsf(h[j].y), r2.y);
+                r2.z = __fmaf_rn(a.inv_k, fabsf(h[j].z), r2.z); r2.w = __fmaf_rn(a.inv_k, fabsf(h[j].w), r2.w);
+            }
+            store4(a.ref2, i0, a.d, r2);
+        }
     }
 }
 
@@ -534,9 +547,10 @@ cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, uint32_t 
     return cudaGetLastError();
 }
 
-cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const FuseBlock* fb, float* ref, int sm_count,
-                           cudaStream_t st, int* launches) {
+cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const FuseBlock* fb, float* ref, float* ref2,
+                           int sm_count, cudaStream_t st, int* launches) {
     CombineArgs a;
+    a.ref2 = ref2; a.inv_k = 1.0f / (float)k;
     for (int j = 0; j < kMaxK; ++j) a.rows[j] = rows[j < k ? j : 0];
     a.alpha = fb->alpha32; a.ref = ref; a.d = d;
     const uint64_t ngroups = (d + 3) / 4;

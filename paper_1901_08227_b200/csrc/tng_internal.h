@@ -49,7 +49,8 @@ cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float
                         int* launches);
 cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, uint32_t M, cudaStream_t st,
                          int* launches);
-cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const FuseBlock* fb, float* ref,
+// ref2 (may be nullptr): also write r' = (1/k) sum_j |h_j| (second reference of the combined form)
+cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const FuseBlock* fb, float* ref, float* ref2,
                            int sm_count, cudaStream_t st, int* launches);
 
 // ---- codec (tng_codec.cu) -----------------------------------------------------
@@ -65,12 +66,13 @@ struct RefFusion {
     int k;
     const float* alpha;   // device, k floats
     float* ref_out;       // device, d floats
+    float* ref2_out;      // device, d floats: second reference (combined form), else nullptr
 };
 bool encode_can_fuse_reference(const CodecGeom& g);
-cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref,
+cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref, const float* ref2,
                           const RefFusion* fusion, uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp,
                           FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
-cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref,
+cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref, const float* ref2,
                           float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
 
 }  // namespace tng

@@ -11,7 +11,7 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libtng.so"
 
 CODEC_SIGN1, CODEC_TERN2, CODEC_QSGD4 = 1, 2, 4
-NORM_NONE, NORM_DIFF, NORM_QUOT = 0, 1, 2
+NORM_NONE, NORM_DIFF, NORM_QUOT, NORM_COMB = 0, 1, 2, 3
 SCALE_ABSMAX, SCALE_L2 = 0, 1
 FUSE_AUTO, FUSE_LAST, FUSE_MEAN, FUSE_LSQ, FUSE_HINDSIGHT = 0, 1, 2, 3, 4
 (OPT_BLOCK, OPT_QSGD_LEVELS, OPT_SCALE_KIND, OPT_SEED_LO, OPT_SEED_HI, OPT_FUSE_MODE, OPT_RIDGE, OPT_QUOT_EPS,
