@@ -656,6 +656,31 @@ __device__ __forceinline__ void decode_round(const DecodeSlot* slot, const uint3
     }
 }
 
+// the same with the worker count known at compile time (no loop, constant shared offsets)
+template <int CODEC, int N>
+__device__ __forceinline__ void decode_round_fixed(const DecodeSlot* slot, const int levels, const uint32_t pw, const int lane,
+                                                   float (&acc)[4]) {
+    constexpr int kWords = 4 * CODEC;
+#pragma unroll
+    for (int k = 0; k < N; ++k) {
+        uint32_t w[kWords];
+#pragma unroll
+        for (int q = 0; q < CODEC; ++q) {
+            const uint4 t = slot->cw[k * CODEC + q];
+            w[4 * q + 0] = t.x; w[4 * q + 1] = t.y; w[4 * q + 2] = t.z; w[4 * q + 3] = t.w;
+        }
+        decode_worker<CODEC>(w, slot->sc[k], levels, pw, lane, acc);
+    }
+}
+
+template <int CODEC>
+__device__ __forceinline__ void decode_round_any(const DecodeSlot* slot, const uint32_t n, const int levels, const uint32_t pw,
+                                                 const int lane, float (&acc)[4]) {
+    if (n == 8 && 8 * CODEC <= 32) decode_round_fixed<CODEC, (8 * CODEC <= 32 ? 8 : 1)>(slot, levels, pw, lane, acc);
+    else if (n == 4) decode_round_fixed<CODEC, 4>(slot, levels, pw, lane, acc);
+    else decode_round<CODEC>(slot, n, levels, pw, lane, acc);
+}
+
 template <int CODEC, int NORM>
 __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeArgs a) {
     __shared__ DecodeSlot slots[kDecWarps];
@@ -695,7 +720,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
             if (has_ref2) r2 = *reinterpret_cast<const float4*>(a.ref2 + (Tn * kTile + (uint64_t)lane * 4u));
         }
         float acc[4] = {z, z, z, z};
-        decode_round<CODEC>(slot, n0, a.levels, pw, lane, acc);
+        decode_round_any<CODEC>(slot, n0, a.levels, pw, lane, acc);
         for (uint32_t m0 = kRound; m0 < a.M; m0 += kRound) {         // more workers than one round holds
             uint4 cw2;
             float sc2;

@@ -30,7 +30,6 @@ struct PipeGeom {
     static constexpr uint32_t kStageBytes = ROWS * kRowBytes;
     static constexpr uint32_t kSmemBytes = STAGES * kStageBytes + 1024;   // + barriers, alignment slack
 };
-constexpr int kMaxStages = 4;
 constexpr int kSpinLimit = 1 << 22;          // polls of try_wait (each may itself block briefly)
 
 enum PipeError : uint32_t { kPipeOk = 0, kPipeFullTimeout = 1, kPipeEmptyTimeout = 2 };
@@ -129,34 +128,6 @@ __device__ __forceinline__ PipeSmem pipe_setup(unsigned char* dyn_smem, uint32_t
     }
     __syncthreads();
     return p;
-}
-
-// Same with the stage count and size chosen at launch time (stage_bytes a multiple of 128).
-__device__ __forceinline__ PipeSmem pipe_setup_rt(unsigned char* dyn_smem, uint32_t nstages, uint32_t stage_bytes,
-                                                  uint32_t consumer_arrivals) {
-    PipeSmem p;
-    p.data = (smem_u32(dyn_smem) + 127u) & ~127u;
-    p.bars = p.data + nstages * stage_bytes;
-    if (threadIdx.x == 0) {
-        for (uint32_t s = 0; s < nstages; ++s) {
-            mbar_init(p.full(s), 1);
-            mbar_init(p.empty(s), consumer_arrivals);
-        }
-        mbar_init_fence();
-    }
-    __syncthreads();
-    return p;
-}
-
-__device__ __forceinline__ uint4 lds128u(uint32_t addr) {
-    uint4 v;
-    asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(addr));
-    return v;
-}
-__device__ __forceinline__ float lds32(uint32_t addr) {
-    float v;
-    asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(addr));
-    return v;
 }
 
 // Row source list of one launch: pointer of each row (all 16-byte aligned): first n_pre
