@@ -79,3 +79,43 @@ def test_full_size_round_in_the_benchmark_configuration():
     assert bool(torch.isfinite(out).all())
     assert bool((scales >= 0).all())
     ctx.close()
+
+
+def test_maximum_vector_length():
+    """d = TNG_MAX_COORDS = 2^31 coordinates (8 GiB per vector), one worker, delayed-gradient
+    reference: every index computation at the top of its range.  Windows at the far end of the
+    vector are checked bit for bit against the oracle (which sees the coordinate offset)."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 40 * (1 << 30):
+        pytest.skip("needs about 40 GiB of free device memory")
+    d = 1 << 31
+    dev = "cuda"
+    gen = torch.Generator(device=dev)
+    gen.manual_seed(11)
+    h = torch.empty(d, device=dev).normal_(generator=gen)
+    ctx = tng.Context(d, 1, 1, tng.CODEC_TERN2, tng.NORM_DIFF, block=128, seed_lo=9)
+    ctx.push_reference(h)
+    del h
+    g = torch.empty((1, d), device=dev).normal_(generator=gen)
+    ctx.step(g)                                          # the aggregate goes to the ring only
+    torch.cuda.synchronize()
+    st = ctx.stats()
+    assert st.pipeline_error == 0 and st.nonfinite_scales == 0 and st.rounds == 1
+    codes, scales = ctx.wire()
+    newest = ctx.history(0)
+    with pytest.raises(tng.TngError):
+        tng.Context(d + 1, 1, 1, tng.CODEC_TERN2, tng.NORM_DIFF)
+    # the reference of the round was the pushed vector; it has been overwritten by the aggregate
+    # (K = 1), so regenerate it
+    gen.manual_seed(11)
+    h = torch.empty(d, device=dev).normal_(generator=gen)
+    for i0, n in [(0, 1024), (d - 2048, 2048), ((1 << 30) - 512, 1024), (d - (1 << 20), 1024)]:
+        sl = slice(i0, i0 + n)
+        ref = to_np(h[sl])
+        wc, ws = oracle.encode(to_np(g[:, sl]), ref, tng.NORM_DIFF, tng.CODEC_TERN2, B=128, seed=(9, 0), t=0, coord_offset=i0)
+        t0, t1 = i0 // 128, (i0 + n) // 128
+        assert np.array_equal(to_np(codes[:, t0 * 8:t1 * 8]).view(np.uint32), wc), f"codes differ in window {i0}"
+        assert np.array_equal(to_np(scales[:, t0:t1]).view(np.uint32), ws.view(np.uint32))
+        want = oracle.decode_aggregate(wc, ws, n, ref, tng.NORM_DIFF, tng.CODEC_TERN2, B=128)
+        assert np.array_equal(to_np(newest[sl]).view(np.uint32), want.view(np.uint32)), f"aggregate differs in window {i0}"
+    ctx.close()
