@@ -53,7 +53,7 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 }
 // One poll; the hardware may park the thread for up to kConsumerNapNs while the phase is
 // incomplete, so a waiting warp costs its scheduler almost no issue slots.
-constexpr uint32_t kConsumerNapNs = 500;
+constexpr uint32_t kConsumerNapNs = 50;
 __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     uint32_t ok;
     asm volatile(
@@ -74,7 +74,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
 // Same for the producer thread, which has nothing else to do: each poll may sleep up to
 // `kProducerNapNs` inside the hardware wait, so that its polling does not take issue slots
 // from the compute warps of its scheduler.  Still bounded.
-constexpr uint32_t kProducerNapNs = 2000;
+constexpr uint32_t kProducerNapNs = 200;
 __device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity) {
     for (int i = 0; i < kSpinLimit; ++i) {
         uint32_t ok;

@@ -86,6 +86,28 @@ def test_long_vectors_take_the_staged_kernels(codec, norm, scale_kind, M, d):
     assert_exact(got, want)
 
 
+@pytest.mark.parametrize("codec", CODECS)
+@pytest.mark.parametrize("factor", [1e-28, 1e-33, 1e-38, 3e-42])
+def test_tiny_and_subnormal_scales(codec, factor):
+    # scales around and below 2^-100 (and subnormal ones): the rounding threshold u*R must be the
+    # same correctly rounded product on both sides
+    d, M = 2048 * 9 + 128 * 3 + 50, 4
+    g = workloads.random_grads(3, M, d, device="cuda", ld=round_up4(d))
+    g.mul_(factor)
+    g[1, 128 * 5: 128 * 6] *= 1e6                       # one ordinary-looking block among the tiny ones
+    ref = (g.mean(0) * 0.5).contiguous()
+    ctx = make_ctx(d, M, 1, codec, tng.NORM_DIFF, block=128, seed_lo=1)
+    ctx.encode(g, ref=ref, step=3)
+    codes, scales = ctx.wire()
+    out = torch.empty(d, device="cuda")
+    ctx.decode_aggregate(out, ref=ref)
+    gn, rn = to_np(g), to_np(ref)
+    oc, osc = oracle.encode(gn, rn, tng.NORM_DIFF, codec, B=128, s=7, seed=(1, 0), t=3)
+    assert same_values(to_np(scales), osc) and np.array_equal(codes_np(codes), oc)
+    assert np.array_equal(to_np(out).view(np.uint32), oracle.decode_aggregate(oc, osc, d, rn, tng.NORM_DIFF, codec, B=128, s=7).view(np.uint32))
+    assert oc.any()
+
+
 @pytest.mark.parametrize("s", [1, 2, 3, 4, 5, 6, 7])
 def test_qsgd_levels(s):
     got, want, _ = run_both(3001, 4, tng.CODEC_QSGD4, tng.NORM_DIFF, 128, s=s)
