@@ -125,9 +125,13 @@ tng_status tng_bind_workspace(tng_ctx* ctx, void* dev_ptr, size_t bytes);
 /* ---- the round ------------------------------------------------------------- */
 /* Seed the ring with a vector (Sec. 4.2: "initialise the reference with a full gradient"). */
 tng_status tng_push_reference(tng_ctx* ctx, const float* vec_dev, void* stream);
-/* One round on M gradient rows (row m at grads_dev + m*ld).  Writes the decoded aggregate
- * v_t (d floats) to agg_out_dev if it is not NULL; the aggregate is always stored as the
- * newest ring entry (tng_history(ctx, 0, ...)). */
+/* One round of Algorithm 1 on M gradient rows (row m at grads_dev + m*ld, device memory):
+ * fusion of the reference from the ring (Sec. 3.1, criterion of Prop. 2), r(w_t) = Q[normalised
+ * gradient] (Eq. 2 / Eq. 3 / the combined form, coding of Sec. 3.2), v_t = the average of the
+ * decoded codes with the reference put back, ring <- v_t.  Writes v_t (d floats) to agg_out_dev
+ * if it is not NULL (device memory, caller-owned); v_t is always stored as the newest ring entry
+ * (tng_history(ctx, 0, ...)).  Errors: TNG_ERR_INVALID_ARG (NULL, misaligned, bad ld),
+ * TNG_ERR_ALLOC (workspace), TNG_ERR_CUDA (launch failure). */
 tng_status tng_step(tng_ctx* ctx, const float* grads_dev, uint64_t ld, float* agg_out_dev,
                     void* stream);
 /* Same round for host buffers: copies the M rows to device staging, runs the round, copies the
@@ -152,14 +156,22 @@ tng_status tng_load_state(tng_ctx* ctx, const void* host_buf, size_t bytes, void
 
 /* ---- stage-level entry points (the kernels tng_step launches; tng_step itself folds the
  * reference combine into the encode pass when there is one scale per 128 coordinates) ---------- */
-/* Fusion: Gram/rhs statistics, K x K solve, reference combine -> the context's reference. */
+/* Fusion (Sec. 3.1 pool, criterion C_nz of Prop. 2): statistics G = <h_i,h_j>, c = <h_i, mean g>,
+ * solve (G + ridge tr(G)/k I) alpha = c, combine r = sum_j alpha_j h_j (fp32 fma chain, newest
+ * first) -> the context's reference (tng_reference); alpha, G, c and C_nz through tng_stats.
+ * Ignores the refresh cadence.  grads_dev / ld as in tng_step. */
 tng_status tng_fuse(tng_ctx* ctx, const float* grads_dev, uint64_t ld, void* stream);
-/* Normalise + scale + quantise + pack against ref_dev (NULL = the context's reference).
- * `step` is the Philox step counter to use (tng_step passes the round number). */
+/* Encode (Eq. 2 / Eq. 3 normalisation; Sec. 3.2: R = max|v|, P(nonzero) = |v|/R; Algorithm 1
+ * "compute R, sample z, transmit"): normalise against ref_dev (d floats, device; NULL = the
+ * context's reference), one scale per block, stochastic rounding, bit packing -> the wire
+ * (tng_wire).  `step` is the Philox step counter (tng_step passes the round number).  With
+ * TNG_NORM_COMB the second reference is always the context's own (from the last fusion). */
 tng_status tng_encode(tng_ctx* ctx, const float* grads_dev, uint64_t ld, const float* ref_dev,
                       uint32_t step, void* stream);
-/* Unpack M code streams, dequantise, average, de-normalise against ref_dev (NULL = context's).
- * Writes out_dev (d floats); does not touch the ring. */
+/* Decode + aggregate (Algorithm 1 "the main server averages", with Eq. 2 / Eq. 3's v = ref + r /
+ * ref . r): unpack the M code streams of the wire, v^m = R^m * symbol, a = (sum_m v^m) / M in
+ * fp32 (m ascending), de-normalise against ref_dev (NULL = context's).  Writes out_dev (d floats,
+ * device); does not touch the ring. */
 tng_status tng_decode_aggregate(tng_ctx* ctx, const float* ref_dev, float* out_dev, void* stream);
 
 /* ---- borrowed views (valid until the next call that changes them) ---------- */
