@@ -362,11 +362,18 @@ __device__ bool chol_solve(const double* A, const double* rhs, int n, double* x)
 }
 
 __global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mode, double ridge, int have_rhs) {
+    // the whole warp brings the statistics into shared memory (one round trip to global memory
+    // instead of one per entry); lane 0 then works on the copy and writes the mirrored Gram back
+    __shared__ double sG[kGramDoubles];
+    const bool stats = (mode == TNG_FUSE_LSQ) || (mode == TNG_FUSE_HINDSIGHT);
+    if (stats)
+        for (int i = threadIdx.x; i < kGramDoubles; i += 32) sG[i] = fb->gram[i];
+    __syncwarp();
     if (threadIdx.x != 0) return;
     double alpha[kMaxK];
     for (int j = 0; j < kMaxK; ++j) alpha[j] = 0.0;
     uint32_t fallback = 0;
-    double* G = fb->gram;
+    double* G = sG;
     if (mode == TNG_FUSE_MEAN) {
         const float inv = __fdiv_rn(1.0f, (float)k);
         for (int j = 0; j < k; ++j) alpha[j] = (double)inv;
@@ -374,7 +381,7 @@ __global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mod
         alpha[0] = 1.0;
     } else {
         for (int a = 0; a < k; ++a)   // mirror the upper triangle
-            for (int b = 0; b < a; ++b) G[a * kGramStride + b] = G[b * kGramStride + a];
+            for (int b = 0; b < a; ++b) fb->gram[a * kGramStride + b] = G[a * kGramStride + b] = G[b * kGramStride + a];
         double A[kMaxK * kMaxK], rhs[kMaxK], x[kMaxK];
         bool ok;
         if (mode == TNG_FUSE_LSQ) {
