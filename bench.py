@@ -355,17 +355,70 @@ def run_ours(args, name, cfg):
         dist.destroy_process_group()
 
 
+def run_producers(args):
+    """Side benchmark (not the headline line): the local-gradient producers of the synthetic
+    workloads, each against its own HBM roofline.  Logistic regression at the dense
+    configuration's per-worker shape (n = 2048 samples x d = 65536 features; the gradient needs
+    two passes over the 512 MiB of features: margins, then the transposed product) and the
+    extended Rosenbrock gradient at d = 2^20, M = 32 (reads x and the M noise rows, writes M rows)."""
+    import torch
+
+    from paper_1901_08227_b200 import tng, workloads
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peak, peak_src = measured_hbm_peak()
+    steps, warm = (args.steps or 20), max(args.warmup or 3, 3)
+
+    def timed(fn):
+        for _ in range(warm):
+            fn()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    out = {}
+    n, d = 2048, 65536
+    X = workloads.normal((n, d), 0, 1, dev)
+    b = torch.sign(workloads.normal((n,), 0, 2, dev))
+    w = workloads.normal((d,), 0, 3, dev, std=0.01)
+    grad = torch.empty(d, device=dev)
+    scratch = torch.empty(tng.logistic_scratch_floats(n, d), device=dev)
+    ms = timed(lambda: tng.logistic_grad(X, b, w, 1e-4, grad, scratch))
+    by = 2.0 * n * d * 4
+    out["logistic_grad"] = {"shape": f"n={n}, d={d}", "ms": ms, "algorithmic_bytes": by, "GBps": by / ms / 1e6,
+                            "frac_of_measured": by / ms / 1e6 / peak}
+    del X
+    d3, M3 = 1 << 20, 32
+    x = workloads.rosenbrock_x0(0, d3, dev)
+    noise = workloads.rosenbrock_noise(0, 0, M3, d3, dev)
+    g = torch.empty((M3, d3), device=dev)
+    ms = timed(lambda: tng.rosenbrock_grad(x, noise, g))
+    by = (2.0 * M3 + 1) * d3 * 4
+    out["rosenbrock_grad"] = {"shape": f"d={d3}, M={M3}", "ms": ms, "algorithmic_bytes": by, "GBps": by / ms / 1e6,
+                              "frac_of_measured": by / ms / 1e6 / peak,
+                              "note": "256 MiB per launch: partly served by the 126 MB L2"}
+    print(json.dumps({"workload": "producers", "peak_GBps": peak, "peak_source": peak_src, "steps": steps, "kernels": out}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=None)
     ap.add_argument("--warmup", type=int, default=None)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="c5_dnn_stream", choices=sorted(WORKLOADS))
+    ap.add_argument("--workload", default="c5_dnn_stream", choices=sorted(WORKLOADS) + ["producers"])
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
+    if args.workload == "producers":
+        run_producers(args)
+        return
     cfg = WORKLOADS[args.workload]
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps

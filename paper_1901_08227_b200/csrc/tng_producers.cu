@@ -13,32 +13,38 @@ namespace {
 constexpr int kMaxRowChunks = 64;
 
 // ---- logistic: margins --------------------------------------------------------
-// One warp per sample: z_i = a_i . w; coef_i = -b_i sigma(-b_i z_i); lossrow_i = log(1+exp(-b_i z_i)).
+// One CTA per sample (grid-stride over samples): the 8 warps split the row, so the many small
+// CTAs balance over the SMs whatever n is.  z_i = a_i . w; coef_i = -b_i sigma(-b_i z_i);
+// lossrow_i = log(1+exp(-b_i z_i)).
 template <bool VEC>
 __global__ void __launch_bounds__(256) logistic_margin_kernel(const float* __restrict__ X, const float* __restrict__ b,
                                                               const float* __restrict__ w, uint64_t n, uint64_t d,
                                                               float* __restrict__ coef, float* __restrict__ lossrow) {
-    const int lane = threadIdx.x & 31;
-    const uint64_t nwarps = (uint64_t)gridDim.x * (blockDim.x >> 5);
-    for (uint64_t i = (uint64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < n; i += nwarps) {
+    __shared__ float part[8];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    for (uint64_t i = blockIdx.x; i < n; i += gridDim.x) {
         const float* row = X + i * d;
         float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
         if (VEC) {
             const float4* r4 = reinterpret_cast<const float4*>(row);
             const float4* w4 = reinterpret_cast<const float4*>(w);
-            for (uint64_t j = lane; j < d / 4; j += 32) {
+#pragma unroll 4
+            for (uint64_t j = threadIdx.x; j < d / 4; j += 256) {
                 const float4 x = __ldcs(r4 + j);
                 const float4 ww = __ldg(w4 + j);
                 acc0 = fmaf(x.x, ww.x, acc0); acc1 = fmaf(x.y, ww.y, acc1);
                 acc2 = fmaf(x.z, ww.z, acc2); acc3 = fmaf(x.w, ww.w, acc3);
             }
         } else {
-            for (uint64_t j = lane; j < d; j += 32) acc0 = fmaf(__ldcs(row + j), __ldg(w + j), acc0);
+            for (uint64_t j = threadIdx.x; j < d; j += 256) acc0 = fmaf(__ldcs(row + j), __ldg(w + j), acc0);
         }
         float z = (acc0 + acc1) + (acc2 + acc3);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) z += __shfl_xor_sync(kFullMask, z, off);
-        if (lane == 0) {
+        if (lane == 0) part[warp] = z;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            z = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
             const float bi = b[i];
             const float t = -bi * z;                       // sigma(t), softplus(t), overflow-safe
             float sig, sp;
@@ -54,6 +60,7 @@ __global__ void __launch_bounds__(256) logistic_margin_kernel(const float* __res
             coef[i] = -bi * sig;
             lossrow[i] = sp;
         }
+        __syncthreads();
     }
 }
 
@@ -68,6 +75,7 @@ __global__ void __launch_bounds__(256) logistic_colsum_kernel(const float* __res
     const uint64_t r1 = (r0 + rows_per_chunk < n) ? r0 + rows_per_chunk : n;
     if (VEC) {
         float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll 8
         for (uint64_t i = r0; i < r1; ++i) {
             const float ci = __ldg(coef + i);
             const float4 x = __ldcs(reinterpret_cast<const float4*>(X + i * d + col));
@@ -166,9 +174,14 @@ __global__ void __launch_bounds__(256) sgd_update_kernel(float* __restrict__ w, 
         w[i] = __fsub_rn(w[i], __fmul_rn(eta, v[i]));
 }
 
+// Row chunks of the transposed product: enough CTAs to fill the GPU (4 per SM), and, when a
+// count up to the limit exists, a total that is a multiple of the SM count so that no SM gets
+// one CTA more than another.
 int row_chunks(uint64_t n, uint64_t d, bool vec) {
     const uint64_t colblocks = ((vec ? d / 4 : d) + 255) / 256;
     uint64_t chunks = (592 + colblocks - 1) / colblocks;
+    for (uint64_t c = chunks; c <= (uint64_t)kMaxRowChunks; ++c)
+        if ((colblocks * c) % 148 == 0) { chunks = c; break; }
     if (chunks > (uint64_t)kMaxRowChunks) chunks = kMaxRowChunks;
     if (chunks > n) chunks = n;
     if (chunks < 1) chunks = 1;
@@ -181,8 +194,7 @@ bool vec_ok(const float* X, const float* w, uint64_t d) {
 
 cudaError_t launch_margins(const float* X, const float* b, const float* w, uint64_t n, uint64_t d, float* coef,
                            float* lossrow, cudaStream_t st) {
-    const uint64_t want = (n + 7) / 8;
-    const int grid = (int)(want < 1184 ? (want ? want : 1) : 1184);
+    const int grid = (int)(n < 148 * 64 ? n : 148 * 64);
     if (vec_ok(X, w, d)) logistic_margin_kernel<true><<<grid, 256, 0, st>>>(X, b, w, n, d, coef, lossrow);
     else logistic_margin_kernel<false><<<grid, 256, 0, st>>>(X, b, w, n, d, coef, lossrow);
     return cudaGetLastError();
