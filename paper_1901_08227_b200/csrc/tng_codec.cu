@@ -59,15 +59,6 @@ __device__ __forceinline__ float absmax_nan2(float a, float b) {
     return r;
 }
 
-// One worker's share of one tile.  A scale that is zero, NaN or infinite needs no
-// special case in the quantisers: u*0 < 0, NaN < x and inf < x are all false, and
-// (int)NaN is 0, so every symbol of such a block comes out as the zero symbol.
-// Returns the bit pattern of the scale it used (for the non-finite bookkeeping).
-//
-// The integer/logic pipe is the busy one in this kernel (Philox xors, compares,
-// ballots), so work that can run on the multiplier pipe is put there: addresses are
-// 32 x 32 -> 64 multiply-adds and the uniform's shift is a high multiply.
-// v = g - r (Eq. 2), v = g * (1/den) (Eq. 3), or v = g
 // operands of the normalisation for the lane's four coordinates: a = r (difference and combined
 // forms) or 1/den (quotient form); b = 1/den' (combined form only)
 struct NormOp {
@@ -125,6 +116,12 @@ __device__ __forceinline__ float encode_tile_stat(const float (&v)[4]) {
 
 // Stochastic rounding of the lane's four values with scale R; x = the lane's Philox call,
 // word c for coordinate 4j+c.  The ballots leave every code word of the tile in every lane.
+// A scale that is zero, NaN or infinite needs no special case: u*0 < 0, NaN < x and inf < x
+// are all false, and (int)NaN is 0, so every symbol of such a block is the zero symbol.
+//
+// The integer/logic pipe is the busy one in the encode kernels (Philox xors, compares,
+// ballots), so work that can run on the multiplier pipe is put there: addresses are
+// 32 x 32 -> 64 multiply-adds and the uniform's shift is a high multiply.
 template <int CODEC, bool FULL>
 __device__ __forceinline__ void encode_quantise(const EncodeArgs& a, const float (&v)[4], const float R, const uint4 x,
                                                 const uint32_t valid, uint32_t (&w)[4 * CODEC]) {
