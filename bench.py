@@ -51,12 +51,14 @@ def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True, ref_in_e
     per = {}
     if fuse == "lsq":
         per["dots"] = 4.0 * K + 4.0 * M
-        if ref_in_encode:
-            per["encode"] = 4.0 * K + 4.0 * M + 4.0 + wire
-        else:
-            per["combine"] = 4.0 * K + 4.0
-            per["encode"] = 4.0 * M + 4.0 + wire
+    elif fuse == "hindsight":
+        per["dots"] = 4.0 * K                      # Gram of the ring only
+    combines = fuse != "last"                      # the delayed-gradient reference is a ring slot as it is
+    if combines and ref_in_encode:
+        per["encode"] = 4.0 * K + 4.0 * M + 4.0 + wire
     else:
+        if combines:
+            per["combine"] = 4.0 * K + 4.0
         per["encode"] = 4.0 * M + 4.0 + wire
     per["decode"] = wire + 4.0 + 4.0 + (4.0 if user_out else 0.0)
     return per
@@ -415,11 +417,20 @@ def main():
     ap.add_argument("--e2e-steps", type=int, default=5)
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    # overrides for sweeps over the codec-sweep configuration (not the headline line)
+    ap.add_argument("--d", type=int, default=None)
+    ap.add_argument("--codec", choices=["sign1", "tern2", "qsgd4"], default=None)
+    ap.add_argument("--norm", choices=["none", "diff", "quot"], default=None)
+    ap.add_argument("--fuse", choices=["lsq", "last", "mean", "hindsight"], default=None)
     args = ap.parse_args()
     if args.workload == "producers":
         run_producers(args)
         return
-    cfg = WORKLOADS[args.workload]
+    cfg = dict(WORKLOADS[args.workload])
+    for key in ("d", "codec", "norm", "fuse"):
+        if getattr(args, key) is not None:
+            cfg[key] = getattr(args, key)
+            args.workload = f"{args.workload}+{key}={cfg[key]}"
     if args.impl == "reference":
         args.steps = 3 if args.steps is None else args.steps
         args.warmup = 1 if args.warmup is None else args.warmup
