@@ -200,7 +200,7 @@ def run_reference(args, name, cfg):
     print(json.dumps(line), flush=True)
 
 
-def time_cpu_baseline(cfg, enums, budget_s=12.0):
+def time_cpu_baseline(cfg, enums, limit_s=12.0):
     import oracle
     from paper_1901_08227_b200 import workloads
     norm, codec, fuse = enums
@@ -218,7 +218,7 @@ def time_cpu_baseline(cfg, enums, budget_s=12.0):
         orc.step(g)
         n += 1
         dt = time.perf_counter() - t0
-        if dt > budget_s or n >= 50:
+        if dt > limit_s or n >= 50:
             break
     per = dt / n
     return {"value": M * d_s * 4 / per / 1e9, "unit": UNIT, "cores": oracle.omp_threads(), "kind": "oracle",
