@@ -143,7 +143,7 @@ def config_dict(name, cfg, world):
             "codec": cfg["codec"], "block": cfg["block"], "fusion": cfg["fuse"],
             "stream": "Student-t(nu=3) around an AR(1) mean (rho 0.99), 64 segments with LogUniform(1e-4,1e-1) scales",
             "l2": "inputs exceed L2: every round streams the whole ring and all M gradient rows from HBM",
-            "sharding": "one process per GPU, each rank its own d coordinates" if world > 1 else "single GPU"}
+            "sharding": "one process per GPU, each rank an independent problem of the full size (no data-path collective)" if world > 1 else "single GPU"}
 
 
 def max_over_ranks(value, world, device):
@@ -151,7 +151,7 @@ def max_over_ranks(value, world, device):
     import torch
     import torch.distributed as dist
     t = torch.tensor([float(value)], dtype=torch.float64, device=device)
-    if world > 1:
+    if world > 1 or (dist.is_available() and dist.is_initialized()):
         dist.all_reduce(t, op=dist.ReduceOp.MAX)
     return t.item()
 
@@ -239,7 +239,8 @@ def run_ours(args, name, cfg):
         raise RuntimeError("bench.py needs a CUDA device (there is no CPU fallback)")
     torch.cuda.set_device(local)
     dev = torch.device("cuda", local)
-    if world > 1:
+    launched = world > 1 or "TORCHELASTIC_RUN_ID" in os.environ     # under torchrun, also with one rank
+    if launched:
         dist.init_process_group("nccl", device_id=dev)
     tng.lib()                                       # fail loudly if libtng.so is missing
 
@@ -265,7 +266,7 @@ def run_ours(args, name, cfg):
     torch.cuda.empty_cache()
 
     def barrier():
-        if world > 1:
+        if launched:
             dist.barrier()
         torch.cuda.synchronize()
 
@@ -353,7 +354,7 @@ def run_ours(args, name, cfg):
         }
         print(json.dumps(line), flush=True)
     ctx.close()
-    if world > 1:
+    if launched:
         dist.destroy_process_group()
 
 
