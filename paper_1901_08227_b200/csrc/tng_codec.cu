@@ -74,7 +74,7 @@ __device__ __forceinline__ NormOp make_norm_op(const float4 r, const float4 r2, 
     if (NORM == TNG_NORM_DIFF || NORM == TNG_NORM_COMB) op.a = r;
     if (NORM == TNG_NORM_QUOT || NORM == TNG_NORM_COMB) {
         const float4 den = quot_den4(NORM == TNG_NORM_QUOT ? r : r2, quot_eps);
-        const float4 inv = make_float4(__fdiv_rn(1.0f, den.x), __fdiv_rn(1.0f, den.y), __fdiv_rn(1.0f, den.z), __fdiv_rn(1.0f, den.w));
+        const float4 inv = make_float4(__frcp_rn(den.x), __frcp_rn(den.y), __frcp_rn(den.z), __frcp_rn(den.w));
         if (NORM == TNG_NORM_QUOT) op.a = inv; else op.b = inv;
     }
     return op;
