@@ -174,6 +174,34 @@ tng_status tng_encode(tng_ctx* ctx, const float* grads_dev, uint64_t ld, const f
  * device); does not touch the ring. */
 tng_status tng_decode_aggregate(tng_ctx* ctx, const float* ref_dev, float* out_dev, void* stream);
 
+/* ---- the same round with the workers on different GPUs ------------------------------- */
+/* Algorithm 1 as the paper states it: every server codes its own gradient, the codes are
+ * exchanged, every server decodes the same average.  Here each process (one per GPU) holds a
+ * context of the SAME (d, M, K, codec, options, seed) and the gradient rows of its own workers
+ * m_first .. m_first + m_count - 1; ring, reference and round counter evolve identically on all
+ * of them.  The library does the rank-local work; the two exchanges are the caller's (NCCL):
+ *   tng_fuse_local      statistics of the local rows: Gram of the ring (the same on every rank)
+ *                       and the local SUMS sum_m <h_i, g^m>, sum_m ||g^m||^2
+ *   [all-reduce (sum) of the tng_local_stats block: 17 doubles on the device]
+ *   tng_fuse_finish     divide by M, solve, combine -> the reference (Sec. 3.1 / Prop. 2)
+ *   tng_encode_local    code the local rows as workers m_first.. into THEIR slots of the wire
+ *   [all-gather of the wire: every rank's slots of codes and scales (tng_wire)]
+ *   tng_decode_commit   decode all M workers, average, put the reference back, push into the
+ *                       ring, advance the round counter (the second half of tng_step)
+ * With all M rows on one rank this sequence equals tng_step except that the statistics are
+ * summed in another order (the reference agrees to rounding of the K coefficients) and that the
+ * refresh cadence option is not applied.  The stochastic rounding of worker m depends only on
+ * (seed, m, round, coordinate), so the wire does not depend on how workers are spread. */
+tng_status tng_fuse_local(tng_ctx* ctx, const float* grads_dev, uint64_t ld, uint32_t m_count, void* stream);
+/* Borrowed device pointer to the block to all-reduce (rhs[16], grad_sq) and its length. */
+tng_status tng_local_stats(tng_ctx* ctx, double** sums_dev, size_t* count);
+tng_status tng_fuse_finish(tng_ctx* ctx, void* stream);
+/* step: the Philox step counter; pass the round number (tng_stats' rounds). */
+tng_status tng_encode_local(tng_ctx* ctx, const float* grads_dev, uint64_t ld, uint32_t m_first, uint32_t m_count,
+                            uint32_t step, void* stream);
+/* agg_out_dev may be NULL (the aggregate is the newest ring entry either way). */
+tng_status tng_decode_commit(tng_ctx* ctx, float* agg_out_dev, void* stream);
+
 /* ---- borrowed views (valid until the next call that changes them) ---------- */
 /* Wire: codes[m] at codes_dev + m*words_per_worker (uint32), scales[m] at scales_dev +
  * m*scales_per_worker.  Tile T = coordinates [128T,128T+128) owns 4b words; word c*b+p, bit j,

@@ -196,7 +196,10 @@ struct StageTimer {
 // ---- the stages -----------------------------------------------------------------------
 // `defer` (may be nullptr): when the encode pass can build the reference itself, the combine
 // launch is skipped and *defer describes the combination for launch_encode.
-tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st, StageTimer* tm, RefFusion* defer) {
+// `stats_ready`: the statistics are already in the FuseBlock as sums over ALL workers (rank-local
+// sums added up by the caller); the statistics pass is skipped and the solve divides them by M.
+tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st, StageTimer* tm, RefFusion* defer,
+                   bool stats_ready = false) {
     if (defer) defer->k = 0;
     const int mode = c->effective_mode();
     c->last_mode = mode;
@@ -221,13 +224,13 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
         return TNG_OK;
     }
     const bool need_dots = (mode == TNG_FUSE_LSQ) || (mode == TNG_FUSE_HINDSIGHT);
-    if (need_dots) {
+    if (need_dots && !stats_ready) {
         const float* g = (mode == TNG_FUSE_LSQ) ? grads : nullptr;
-        TNG_CUDA(c, launch_dots(rows, (int)c->k, c->d, g, c->M, ld, c->partials(), c->fb(), c->sm_count, st, &launches));
-        c->last_had_stats = true;
+        TNG_CUDA(c, launch_dots(rows, (int)c->k, c->d, g, c->M, ld, 0, c->partials(), c->fb(), c->sm_count, st, &launches));
     }
-    if (tm) tm->mark(0, need_dots);
-    TNG_CUDA(c, launch_solve(c->fb(), (int)c->k, mode, c->ridge, c->M, st, &launches));
+    c->last_had_stats = need_dots;
+    if (tm) tm->mark(0, need_dots && !stats_ready);
+    TNG_CUDA(c, launch_solve(c->fb(), (int)c->k, mode, c->ridge, (stats_ready && mode == TNG_FUSE_LSQ) ? (double)c->M : 1.0, st, &launches));
     c->last_solved = true;
     if (tm) tm->mark(1, true);
     if (defer && encode_can_fuse_reference(c->geom)) {
@@ -250,7 +253,7 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
 tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* ref, const RefFusion* fusion, uint32_t step,
                      cudaStream_t st) {
     int launches = 0;
-    TNG_CUDA(c, launch_encode(c->geom, grads, ld, ref, c->ref2_buf(), fusion, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
+    TNG_CUDA(c, launch_encode(c->geom, 0, grads, ld, ref, c->ref2_buf(), fusion, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
                               c->fb(), c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
@@ -260,6 +263,18 @@ tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, c
     int launches = 0;
     TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), ref, c->ref2_buf(), out_a, out_b, c->fb(), c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
+    return TNG_OK;
+}
+
+// The decoded aggregate goes straight into the next ring slot (and to the caller's buffer); the
+// round is then complete: ring rotated, round counter advanced.
+tng_status decode_commit(tng_ctx* c, float* out, cudaStream_t st) {
+    const int slot = (c->k == 0) ? c->head : (c->head + 1) % (int)c->K;
+    tng_status s = do_decode(c, c->ref_cur, c->ring(slot), out, st);
+    if (s != TNG_OK) return s;
+    c->head = slot;
+    if (c->k < c->K) c->k += 1;
+    c->rounds += 1;
     return TNG_OK;
 }
 
@@ -282,14 +297,9 @@ tng_status step_impl(tng_ctx* c, const float* grads, uint64_t ld, float* out, cu
     s = do_encode(c, grads, ld, c->ref_cur, &fusion, (uint32_t)c->rounds, st);
     if (s != TNG_OK) return s;
     tm.mark(3, true);
-    // the decoded aggregate goes straight into the next ring slot (and to the caller's buffer)
-    const int slot = (c->k == 0) ? c->head : (c->head + 1) % (int)c->K;
-    s = do_decode(c, c->ref_cur, c->ring(slot), out, st);
+    s = decode_commit(c, out, st);
     if (s != TNG_OK) return s;
     tm.mark(4, true);
-    c->head = slot;
-    if (c->k < c->K) c->k += 1;
-    c->rounds += 1;
     return TNG_OK;
 }
 
@@ -505,6 +515,73 @@ tng_status tng_load_state(tng_ctx* c, const void* host_buf, size_t bytes, void* 
     c->last_had_stats = false;
     c->last_solved = false;
     return TNG_OK;
+}
+
+// ---- one worker (or a few) per GPU: the rank-local pieces of a round ---------------------
+tng_status tng_fuse_local(tng_ctx* c, const float* grads_dev, uint64_t ld, uint32_t m_count, void* stream) {
+    if (!c || m_count < 1 || m_count > c->M) return TNG_ERR_INVALID_ARG;
+    tng_status s = check_rows(c, grads_dev, ld);
+    if (s != TNG_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    // the block the caller adds up over the ranks: rhs[16] and grad_sq; zero when this mode has none
+    TNG_CUDA(c, cudaMemsetAsync(c->fb()->gram + kGramRhs, 0, (kMaxK + 1) * sizeof(double), st));
+    const int mode = c->effective_mode();
+    if (c->k == 0 || (mode != TNG_FUSE_LSQ && mode != TNG_FUSE_HINDSIGHT)) return TNG_OK;
+    const float* rows[kMaxK];
+    for (uint32_t j = 0; j < c->k; ++j) rows[j] = c->ring(c->hist_slot(j));
+    int launches = 0;
+    TNG_CUDA(c, launch_dots(rows, (int)c->k, c->d, mode == TNG_FUSE_LSQ ? grads_dev : nullptr, m_count, ld, 1, c->partials(), c->fb(),
+                            c->sm_count, st, &launches));
+    c->launches += (uint64_t)launches;
+    return TNG_OK;
+}
+
+tng_status tng_local_stats(tng_ctx* c, double** sums_dev, size_t* count) {
+    if (!c || !sums_dev || !count) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready) return TNG_ERR_STATE;
+    *sums_dev = c->fb()->gram + kGramRhs;
+    *count = (size_t)kMaxK + 1;
+    return TNG_OK;
+}
+
+tng_status tng_fuse_finish(tng_ctx* c, void* stream) {
+    if (!c) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready) return TNG_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    return do_fuse(c, nullptr, 0, st, nullptr, nullptr, true);
+}
+
+tng_status tng_encode_local(tng_ctx* c, const float* grads_dev, uint64_t ld, uint32_t m_first, uint32_t m_count, uint32_t step,
+                            void* stream) {
+    if (!c || m_count < 1 || m_first >= c->M || m_count > c->M - m_first) return TNG_ERR_INVALID_ARG;
+    tng_status s = check_rows(c, grads_dev, ld);
+    if (s != TNG_OK) return s;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    if (!c->ref_cur && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;   // no fusion has produced a reference yet
+    if (c->norm == TNG_NORM_COMB && !c->ref2_valid) return TNG_ERR_STATE;
+    CodecGeom g = c->geom;
+    g.M = m_count;
+    int launches = 0;
+    TNG_CUDA(c, launch_encode(g, m_first, grads_dev, ld, c->ref_cur, c->ref2_buf(), nullptr, step, c->codes() + (size_t)m_first * g.wpw,
+                              c->scales() + (size_t)m_first * g.nblk, c->tile_stat(), c->tree(), c->fb(), c->sm_count, st, &launches));
+    c->launches += (uint64_t)launches;
+    return TNG_OK;
+}
+
+tng_status tng_decode_commit(tng_ctx* c, float* agg_out_dev, void* stream) {
+    if (!c || (agg_out_dev && !aligned16(agg_out_dev))) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready) return TNG_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    if (!c->ref_cur && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;
+    return decode_commit(c, agg_out_dev, st);
 }
 
 tng_status tng_fuse(tng_ctx* c, const float* grads_dev, uint64_t ld, void* stream) {

@@ -35,6 +35,7 @@ struct EncodeArgs {
     uint64_t tile_begin;   // first tile this launch handles (the staged kernel takes the ones before it)
     uint32_t ld, nblk, wpw;
     uint32_t M, step;
+    uint32_t m_base;   // worker index of row 0 (Philox counter word); the wire pointers are already offset
     uint32_t pow24;    // 1 << 24 as a run-time value: x >> 8 is taken as umulhi(x, 2^24)
     uint32_t rk[20];   // Philox round keys (key + r * Weyl), computed once on the host
     int levels;
@@ -189,7 +190,7 @@ __device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const flo
     uint32_t w[kWords];
     float R;
     uint4 x = make_uint4(0u, 0u, 0u, 0u);
-    if (PHASE != kPhaseStat) x = philox4x32_10_rk(q_lo, q_hi, m, a.step, a.rk);
+    if (PHASE != kPhaseStat) x = philox4x32_10_rk(q_lo, q_hi, a.m_base + m, a.step, a.rk);
     if (!encode_symbols<CODEC, NORM, SCALE, PHASE, FULL>(a, g, op, m, T, x, blk, lane, valid, w, R)) return 0u;
     if (lane == 0) {
         uint4* dst = reinterpret_cast<uint4*>(a.codes + ((uint64_t)m * a.wpw + T * (uint64_t)kWords));
@@ -415,7 +416,7 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
 #pragma unroll
                 for (int k0 = 0; k0 < G::kRows; k0 += kPhiloxBatch) {
                     uint4 x[kPhiloxBatch];
-                    philox4x32_10_rk_batch<kPhiloxBatch>(q_lo, q_hi, m0 + k0, a.step, a.rk, x);
+                    philox4x32_10_rk_batch<kPhiloxBatch>(q_lo, q_hi, a.m_base + m0 + k0, a.step, a.rk, x);
 #pragma unroll
                     for (int kk = 0; kk < kPhiloxBatch; ++kk) {
                         const int k = k0 + kk;
@@ -432,7 +433,7 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                     const float4 g = *reinterpret_cast<const float4*>(base + k * G::kRowBytes);
                     uint32_t w[kWords];
                     float R;
-                    const uint4 x = philox4x32_10_rk(q_lo, q_hi, m0 + k, a.step, a.rk);
+                    const uint4 x = philox4x32_10_rk(q_lo, q_hi, a.m_base + m0 + k, a.step, a.rk);
                     encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, x, T, lane, 0xFu, w, R);
                     store_words_if<CODEC>((uint32_t)lane == k, my_codes, w);
                     my_R = ((uint32_t)lane == k) ? R : my_R;
@@ -889,7 +890,7 @@ size_t tree_tmp_floats(const CodecGeom& g) {
 
 bool encode_can_fuse_reference(const CodecGeom& g) { return g.block == kTile && g.norm != TNG_NORM_NONE; }
 
-cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref, const float* ref2,
+cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grads, uint64_t ld, const float* ref, const float* ref2,
                           const RefFusion* fusion,
                           uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp, FuseBlock* fb,
                           int sm_count, cudaStream_t st, int* launches) {
@@ -905,7 +906,7 @@ cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, c
     a.grads = grads; a.ref = ref; a.codes = codes; a.scales = scales; a.tile_stat = tile_stat;
     a.nonfinite = &fb->nonfinite; a.pipe_error = &fb->pipe_error; a.tile_begin = 0;
     a.ld = (uint32_t)ld; a.d = g.d; a.ntile = g.ntile; a.nblk = (uint32_t)g.nblk; a.block = g.block; a.wpw = (uint32_t)g.wpw;
-    a.M = g.M; a.step = step; a.levels = g.levels; a.pow24 = 1u << 24;
+    a.M = g.M; a.step = step; a.m_base = m_base; a.levels = g.levels; a.pow24 = 1u << 24;
     a.quot_eps = g.quot_eps;
     philox_round_keys(g.seed_lo, g.seed_hi, a.rk);
     cudaError_t e;

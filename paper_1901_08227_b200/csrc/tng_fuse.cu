@@ -28,6 +28,7 @@ struct DotsArgs {
     FuseBlock* fb;
     uint64_t d, ld;
     uint32_t M;
+    uint32_t divisor;         // rhs and grad_sq are divided by this (M for means, 1 for raw sums)
     short dst[kDotsMaxAcc];   // destination of accumulator i inside fb->gram
 };
 
@@ -74,7 +75,7 @@ __device__ __forceinline__ void dots_finish(const double (&acc)[kAcc], const Dot
     if (tid < kAcc) {
         double v = 0.0;
         for (uint32_t b = 0; b < gridDim.x; ++b) v += __ldcg(a.partials + (uint64_t)b * kDotsMaxAcc + tid);
-        if (SAME && tid >= kPairs) v /= (double)a.M;   // rhs and grad_sq use the mean
+        if (SAME && tid >= kPairs) v /= (double)a.divisor;   // rhs and grad_sq: mean over the rows, or raw sums
         if (!(SAME && !with_g && tid >= kPairs)) a.fb->gram[a.dst[tid]] = v;
     }
     if (tid == 0) a.fb->dots_arrivals = 0;   // ready for the next launch on this stream
@@ -361,13 +362,20 @@ __device__ bool chol_solve(const double* A, const double* rhs, int n, double* x)
     return true;
 }
 
-__global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mode, double ridge, int have_rhs) {
+__global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mode, double ridge, int have_rhs, double rhs_div) {
     // the whole warp brings the statistics into shared memory (one round trip to global memory
     // instead of one per entry); lane 0 then works on the copy and writes the mirrored Gram back
     __shared__ double sG[kGramDoubles];
     const bool stats = (mode == TNG_FUSE_LSQ) || (mode == TNG_FUSE_HINDSIGHT);
     if (stats)
-        for (int i = threadIdx.x; i < kGramDoubles; i += 32) sG[i] = fb->gram[i];
+        for (int i = threadIdx.x; i < kGramDoubles; i += 32) {
+            double v = fb->gram[i];
+            if (rhs_div != 1.0 && i >= kGramRhs) {   // sums over all workers -> means
+                v /= rhs_div;
+                fb->gram[i] = v;
+            }
+            sG[i] = v;
+        }
     __syncwarp();
     if (threadIdx.x != 0) return;
     double alpha[kMaxK];
@@ -492,13 +500,14 @@ cudaError_t combine_k(const CombineArgs& a, int grid, cudaStream_t st) {
 }  // namespace
 
 cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float* grads, uint32_t M, uint64_t ld,
-                        double* partials, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
+                        uint32_t divisor, double* partials, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
     const uint64_t ngroups = (d + 3) / 4;
     uint64_t want = (ngroups + kDotsThreads - 1) / kDotsThreads;
     if (want < 1) want = 1;
     const int grid = (int)(want < (uint64_t)sm_count ? want : (uint64_t)sm_count);
     DotsArgs a;
     a.grads = grads; a.partials = partials; a.fb = fb; a.d = d; a.ld = ld; a.M = M;
+    a.divisor = divisor ? divisor : M;
     cudaError_t e = cudaSuccess;
     // long vectors, at most 8 history rows: the staged kernel
     if (k <= 8 && d >= kDotsPipeMinCoords) {
@@ -547,9 +556,8 @@ cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float
     return e;
 }
 
-cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, uint32_t M, cudaStream_t st, int* launches) {
-    (void)M;
-    solve_kernel<<<1, 32, 0, st>>>(fb, k, mode, ridge, mode == TNG_FUSE_LSQ ? 1 : 0);
+cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, double rhs_div, cudaStream_t st, int* launches) {
+    solve_kernel<<<1, 32, 0, st>>>(fb, k, mode, ridge, mode == TNG_FUSE_LSQ ? 1 : 0, rhs_div);
     ++*launches;
     return cudaGetLastError();
 }

@@ -44,10 +44,13 @@ struct CodecGeom {
 // ---- fusion (tng_fuse.cu) ---------------------------------------------------
 // rows[j] = h_{j+1}.  Accumulates G (and with grads != nullptr the rhs and grad_sq)
 // into fb->gram via per-CTA partials in `partials` (kDotsMaxCtas * kDotsMaxAcc doubles).
+// divisor: what the gradient sums (rhs, grad_sq) are divided by; 0 = M (the mean over the rows
+// given), 1 = raw sums (a caller that adds the sums of several GPUs divides later, in the solve).
 cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float* grads, uint32_t M,
-                        uint64_t ld, double* partials, FuseBlock* fb, int sm_count, cudaStream_t st,
+                        uint64_t ld, uint32_t divisor, double* partials, FuseBlock* fb, int sm_count, cudaStream_t st,
                         int* launches);
-cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, uint32_t M, cudaStream_t st,
+// rhs_div: the solve first divides rhs and grad_sq by it (1 = they are means already).
+cudaError_t launch_solve(FuseBlock* fb, int k, int mode, double ridge, double rhs_div, cudaStream_t st,
                          int* launches);
 // ref2 (may be nullptr): also write r' = (1/k) sum_j |h_j| (second reference of the combined form)
 cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const FuseBlock* fb, float* ref, float* ref2,
@@ -69,7 +72,9 @@ struct RefFusion {
     float* ref2_out;      // device, d floats: second reference (combined form), else nullptr
 };
 bool encode_can_fuse_reference(const CodecGeom& g);
-cudaError_t launch_encode(const CodecGeom& g, const float* grads, uint64_t ld, const float* ref, const float* ref2,
+// The g.M rows at `grads` are workers m_base .. m_base + g.M - 1 (their Philox streams); codes and
+// scales point at the wire slot of worker m_base.
+cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grads, uint64_t ld, const float* ref, const float* ref2,
                           const RefFusion* fusion, uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp,
                           FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
 cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref, const float* ref2,

@@ -78,7 +78,7 @@ extern "C" tng_status tng_gram_static(const float* const* rows_dev, uint32_t k, 
     // the array keeps whatever the last call left: the arrival counter must start at zero
     if (cudaMemsetAsync(fb, 0, sizeof(FuseBlock), st) != cudaSuccess) return TNG_ERR_CUDA;
     int launches = 0;
-    if (tng::launch_dots(rows_dev, (int)k, d, grads_dev, M, ld, partials, fb, g_sm_count[dev], st, &launches) != cudaSuccess)
+    if (tng::launch_dots(rows_dev, (int)k, d, grads_dev, M, ld, 0, partials, fb, g_sm_count[dev], st, &launches) != cudaSuccess)
         return TNG_ERR_CUDA;
     pack_static_gram_kernel<<<1, 128, 0, st>>>((int)k, out_dev);
     return cudaGetLastError() == cudaSuccess ? TNG_OK : TNG_ERR_CUDA;

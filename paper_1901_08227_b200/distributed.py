@@ -1,0 +1,58 @@
+"""Workers spread over GPUs: one process per GPU (``torch.distributed``, NCCL), every process a
+``tng.Context`` of the same configuration and the gradient rows of its own workers.
+
+A round is the rank-local stages of the library with two exchanges between them (Algorithm 1:
+every server codes its gradient, the codes are exchanged, everyone decodes the same average):
+
+    fuse_local -> all-reduce of 17 doubles -> fuse_finish -> encode_local
+               -> all-gather of the wire (codes and scales) -> decode_commit
+
+Only plumbing lives here; every computation is a library call.  The collectives run on the
+wire and statistics buffers in place (zero-copy views of the context's workspace), which are
+this GPU's own memory.
+"""
+from __future__ import annotations
+
+import torch
+import torch.distributed as dist
+
+from . import tng
+
+
+def worker_range(rank: int, world: int, M: int):
+    """Workers [first, first + count) of `rank`: M must split evenly over the ranks so that the
+    wire can be all-gathered as equal blocks."""
+    if M % world != 0:
+        raise ValueError(f"M = {M} workers do not split evenly over {world} ranks")
+    count = M // world
+    return rank * count, count
+
+
+class DistributedRound:
+    """Drives one context per rank.  `group` may be None (a single process: no exchange)."""
+
+    def __init__(self, ctx: tng.Context, group=None):
+        self.ctx, self.group = ctx, group
+        self.world = dist.get_world_size(group) if group is not None else 1
+        self.rank = dist.get_rank(group) if group is not None else 0
+        self.first, self.count = worker_range(self.rank, self.world, ctx.M)
+        self.round = 0
+
+    def step(self, local_grads: torch.Tensor, out: torch.Tensor | None = None):
+        """local_grads: (count, d) rows of this rank's workers.  Returns `out` (the aggregate)."""
+        if local_grads.shape[0] != self.count:
+            raise ValueError(f"rank {self.rank} owns {self.count} workers, got {local_grads.shape[0]} rows")
+        ctx = self.ctx
+        ctx.fuse_local(local_grads)
+        if self.world > 1:
+            dist.all_reduce(ctx.local_stats(), op=dist.ReduceOp.SUM, group=self.group)
+        ctx.fuse_finish()
+        ctx.encode_local(local_grads, self.first, self.round)
+        if self.world > 1:
+            codes, scales = ctx.wire_views()
+            lo, hi = self.first, self.first + self.count
+            dist.all_gather_into_tensor(codes, codes[lo:hi].clone(), group=self.group)
+            dist.all_gather_into_tensor(scales, scales[lo:hi].clone(), group=self.group)
+        ctx.decode_commit(out)
+        self.round += 1
+        return out

@@ -27,6 +27,7 @@ EXPORTS = [
     "tng_wire", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
     "tng_logistic_scratch_floats", "tng_logistic_grad", "tng_logistic_loss", "tng_rosenbrock_grad",
     "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static", "tng_state_bytes", "tng_save_state", "tng_load_state",
+    "tng_fuse_local", "tng_local_stats", "tng_fuse_finish", "tng_encode_local", "tng_decode_commit",
 ]
 
 
@@ -89,6 +90,11 @@ def lib():
         L.tng_state_bytes.argtypes = [vp, C.POINTER(C.c_size_t)]
         L.tng_save_state.argtypes = [vp, vp, C.c_size_t, C.POINTER(C.c_size_t), vp]
         L.tng_load_state.argtypes = [vp, vp, C.c_size_t, vp]
+        L.tng_fuse_local.argtypes = [vp, vp, u64, u32, vp]
+        L.tng_local_stats.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
+        L.tng_fuse_finish.argtypes = [vp, vp]
+        L.tng_encode_local.argtypes = [vp, vp, u64, u32, u32, u32, vp]
+        L.tng_decode_commit.argtypes = [vp, vp, vp]
         L.tng_gram_static.argtypes = [C.POINTER(vp), u32, u64, vp, u32, u64, vp, vp]
         _lib = L
     return _lib
@@ -203,6 +209,33 @@ class Context:
             raise TypeError("state must be a contiguous host uint8 tensor")
         _check(lib().tng_load_state(self._h, buf.data_ptr(), buf.numel(), _stream()), "tng_load_state")
 
+    # -- rank-local stages (workers spread over several GPUs)
+    def fuse_local(self, grads):
+        p, ld = _rows(grads)
+        _check(lib().tng_fuse_local(self._h, p, ld, grads.shape[0], _stream()), "tng_fuse_local")
+
+    def local_stats(self) -> torch.Tensor:
+        """Zero-copy float64 view of the block to all-reduce (sum) between fuse_local and fuse_finish."""
+        p, n = C.c_void_p(), C.c_size_t()
+        _check(lib().tng_local_stats(self._h, C.byref(p), C.byref(n)), "tng_local_stats")
+        return _view(p.value, (n.value,), torch.float64)
+
+    def fuse_finish(self):
+        _check(lib().tng_fuse_finish(self._h, _stream()), "tng_fuse_finish")
+
+    def encode_local(self, grads, m_first, step):
+        p, ld = _rows(grads)
+        _check(lib().tng_encode_local(self._h, p, ld, int(m_first), grads.shape[0], int(step), _stream()), "tng_encode_local")
+
+    def decode_commit(self, out=None):
+        _check(lib().tng_decode_commit(self._h, _dev(out), _stream()), "tng_decode_commit")
+        return out
+
+    def wire_views(self):
+        """Zero-copy views of the wire, (M, words) int32 codes and (M, scales) float32, for collectives."""
+        cp, wpw, sp, spw = self.wire_pointers()
+        return _view(cp, (self.M, wpw), torch.int32), _view(sp, (self.M, spw), torch.float32)
+
     def fuse(self, grads):
         p, ld = _rows(grads)
         _check(lib().tng_fuse(self._h, p, ld, _stream()), "tng_fuse")
@@ -260,7 +293,7 @@ class _DeviceView:
 
 
 def _view(ptr, shape, dtype):
-    typestr = {torch.float32: "<f4", torch.int32: "<i4"}[dtype]
+    typestr = {torch.float32: "<f4", torch.int32: "<i4", torch.float64: "<f8"}[dtype]
     return torch.as_tensor(_DeviceView(ptr, shape, typestr), device="cuda")
 
 

@@ -70,3 +70,32 @@ def test_algorithmic_bytes_of_the_round():
     assert sum(per.values()) == 148.5
     split = bench.algorithmic_bytes_per_coord(8, 8, 2, 128, "lsq", ref_in_encode=False)
     assert split["combine"] == 36.0 and split["encode"] == 38.25
+
+
+def _gather_main(rank, world, port, out_dir):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_1901_08227_b200 import distributed
+    M, words = 6, 10
+    first, count = distributed.worker_range(rank, world, M)
+    wire = torch.zeros((M, words), dtype=torch.int32)
+    wire[first:first + count] = torch.arange(first * words, (first + count) * words, dtype=torch.int32).view(count, words)
+    dist.all_gather_into_tensor(wire, wire[first:first + count].clone())     # as DistributedRound does, in place
+    stats = torch.full((17,), float(rank + 1), dtype=torch.float64)
+    dist.all_reduce(stats)
+    Path(out_dir, f"wire{rank}.json").write_text(json.dumps({"wire": wire.tolist(), "stats": stats.tolist(), "range": [first, count]}))
+    dist.destroy_process_group()
+
+
+def test_the_wire_exchange_assembles_every_worker_slot_on_every_rank(tmp_path):
+    world = 2
+    mp.spawn(_gather_main, args=(world, _free_port(), str(tmp_path)), nprocs=world, join=True)
+    r = [json.loads((tmp_path / f"wire{i}.json").read_text()) for i in range(world)]
+    want = np.arange(60).reshape(6, 10).tolist()
+    assert r[0]["wire"] == want and r[1]["wire"] == want          # worker m's words in slot m everywhere
+    assert r[0]["stats"] == [3.0] * 17 and r[1]["stats"] == [3.0] * 17
+    assert r[0]["range"] == [0, 3] and r[1]["range"] == [3, 3]
+    from paper_1901_08227_b200 import distributed
+    import pytest
+    with pytest.raises(ValueError):
+        distributed.worker_range(0, 4, 6)
