@@ -529,20 +529,33 @@ __device__ __forceinline__ void decode_worker(const uint32_t (&w)[4 * CODEC], co
     const uint32_t Re = ok ? __float_as_uint(R) : 0u;
     const uint32_t okm = ok ? 0x80000000u : 0u;
     if (CODEC == TNG_CODEC_TERN2) {
-#pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            // sign plane -> sign bit of R; the add is skipped for the zero symbol (acc + 0 == acc).
-            // Written out so that it stays four instructions: a logic op that also sets the
-            // predicate, a multiply (bit -> sign position), a three-input logic op, a predicated add.
-            asm("{\n\t.reg .pred p, pt;\n\t.reg .b32 t, s;\n\t"
-                "setp.eq.u32 pt, 0, 0;\n\t"
-                "lop3.and.b32 t|p, %1, %3, %3, 0xC0, pt;\n\t"   // p = (nonzero word & lane bit) != 0
-                "mul.lo.u32 s, %2, %4;\n\t"                      // lane's sign bit -> bit 31
-                "lop3.b32 s, s, %5, %6, 0x6A;\n\t"              // (s & okm) ^ Re
-                "@p add.rn.f32 %0, %0, s;\n\t}"
-                : "+f"(acc[c])
-                : "r"(w[c * 2]), "r"(w[c * 2 + 1]), "r"(1u << lane), "r"(pw), "r"(okm), "r"(Re));
-        }
+        // Per coordinate: the lane's bit of the non-zero plane decides whether anything is added
+        // (acc + 0 == acc, and an unusable scale adds nothing either: the predicate is and-ed with
+        // `ok`); the lane's bit of the sign plane, moved to bit 31 by a multiply, flips the sign of R.
+        // Written out so that it stays four instructions per coordinate: a logic op that sets the
+        // predicate, a multiply, a three-input logic op ((s & 0x80000000) ^ R), a predicated add.
+        constexpr int kT = (CODEC == TNG_CODEC_TERN2) ? 2 : 0;   // plane stride (keeps indices in range elsewhere)
+        asm("{\n\t.reg .pred p, pk;\n\t.reg .b32 t, s;\n\t"
+            "setp.ne.u32 pk, %12, 0;\n\t"
+            "lop3.and.b32 t|p, %4, %13, %13, 0xC0, pk;\n\t"
+            "mul.lo.u32 s, %5, %14;\n\t"
+            "lop3.b32 s, s, 0x80000000, %15, 0x6A;\n\t"
+            "@p add.rn.f32 %0, %0, s;\n\t"
+            "lop3.and.b32 t|p, %6, %13, %13, 0xC0, pk;\n\t"
+            "mul.lo.u32 s, %7, %14;\n\t"
+            "lop3.b32 s, s, 0x80000000, %15, 0x6A;\n\t"
+            "@p add.rn.f32 %1, %1, s;\n\t"
+            "lop3.and.b32 t|p, %8, %13, %13, 0xC0, pk;\n\t"
+            "mul.lo.u32 s, %9, %14;\n\t"
+            "lop3.b32 s, s, 0x80000000, %15, 0x6A;\n\t"
+            "@p add.rn.f32 %2, %2, s;\n\t"
+            "lop3.and.b32 t|p, %10, %13, %13, 0xC0, pk;\n\t"
+            "mul.lo.u32 s, %11, %14;\n\t"
+            "lop3.b32 s, s, 0x80000000, %15, 0x6A;\n\t"
+            "@p add.rn.f32 %3, %3, s;\n\t}"
+            : "+f"(acc[0]), "+f"(acc[1]), "+f"(acc[2]), "+f"(acc[3])
+            : "r"(w[0]), "r"(w[kT ? 1 : 0]), "r"(w[1 * kT]), "r"(w[1 * kT + (kT ? 1 : 0)]), "r"(w[2 * kT]), "r"(w[2 * kT + (kT ? 1 : 0)]),
+              "r"(w[3 * kT]), "r"(w[3 * kT + (kT ? 1 : 0)]), "r"((uint32_t)ok), "r"(1u << lane), "r"(pw), "r"(__float_as_uint(R)));
     } else if (CODEC == TNG_CODEC_SIGN1) {
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
