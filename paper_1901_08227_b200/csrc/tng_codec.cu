@@ -392,7 +392,6 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
         // ---- the gradient rows, one fill of up to 8 workers at a time.  Every lane ends up with
         // all words of every worker; lane k writes worker k of the fill through a pointer it
         // computes once per fill, and the fill's scales go out as one store.
-        uint32_t rmax = 0;
         constexpr int kWords = 4 * CODEC;
         for (uint32_t m0 = 0; m0 < M; m0 += G::kRows) {
             const uint32_t s = it % G::kStages, use = it / G::kStages;
@@ -425,7 +424,6 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                         encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g[k], op, m0 + k, T, x[kk], T, lane, 0xFu, w, R);
                         store_words_if<CODEC>(lane == k, my_codes, w);
                         my_R = (lane == k) ? R : my_R;
-                        rmax = max(rmax, __float_as_uint(R));
                     }
                 }
             } else {
@@ -437,20 +435,16 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                     encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, x, T, lane, 0xFu, w, R);
                     store_words_if<CODEC>((uint32_t)lane == k, my_codes, w);
                     my_R = ((uint32_t)lane == k) ? R : my_R;
-                    rmax = max(rmax, __float_as_uint(R));
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pipe.empty(s));   // this warp has read the stage
             }
-            if (lane < G::kRows && mine < M) a.scales[(uint64_t)mine * a.nblk + T] = my_R;
+            const bool writes = lane < G::kRows && mine < M;
+            if (writes) a.scales[(uint64_t)mine * a.nblk + T] = my_R;
+            // NaN or +inf scales (rare) are counted from the lanes that hold them
+            const uint32_t bad = __ballot_sync(kFullMask, writes && __float_as_uint(my_R) >= 0x7f800000u);
+            if (bad != 0u && lane == 0) atomicAdd(a.nonfinite, (unsigned long long)__popc(bad));
             ++it;
-        }
-        __syncwarp();
-        // NaN or +inf scales are rare: only then count them, from the scales just written
-        if (rmax >= 0x7f800000u && lane == 0) {
-            unsigned long long bad = 0;
-            for (uint32_t m = 0; m < M; ++m) bad += (__float_as_uint(a.scales[(uint64_t)m * a.nblk + T]) >= 0x7f800000u) ? 1ull : 0ull;
-            atomicAdd(a.nonfinite, bad);
         }
     }
 }
