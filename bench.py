@@ -67,7 +67,7 @@ def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True, ref_in_e
 # dram__bytes_read.sum + dram__bytes_write.sum per coordinate of the dominant kernel, from the ncu
 # capture summarised under profiles/ (taken at d = 2^24 and scaled by d: every kernel streams each
 # coordinate once).  None = the kernel changed after the capture.
-NCU_TRAFFIC_BYTES_PER_COORD = {"encode": 69.96, "dots": 64.33, "decode": 11.24}
+NCU_TRAFFIC_BYTES_PER_COORD = {"encode": 69.92, "dots": 64.35, "decode": 11.16}
 
 
 def measured_hbm_peak():
