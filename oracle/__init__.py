@@ -24,7 +24,7 @@ _HDR = _HERE / "tng_oracle.h"
 _LIB = _HERE / "libtng_oracle.so"
 
 CODEC_SIGN1, CODEC_TERN2, CODEC_QSGD4 = 1, 2, 4
-NORM_NONE, NORM_DIFF, NORM_QUOT, NORM_COMB = 0, 1, 2, 3
+NORM_NONE, NORM_DIFF, NORM_QUOT, NORM_COMB, NORM_MEAN = 0, 1, 2, 3, 4
 SCALE_ABSMAX, SCALE_L2 = 0, 1
 FUSE_AUTO, FUSE_LAST, FUSE_MEAN, FUSE_LSQ, FUSE_HINDSIGHT = 0, 1, 2, 3, 4
 OPT_BLOCK, OPT_QSGD_LEVELS, OPT_SCALE_KIND, OPT_SEED_LO, OPT_SEED_HI, OPT_FUSE_MODE, OPT_RIDGE, OPT_QUOT_EPS, OPT_REF_EVERY = range(9)
@@ -70,13 +70,17 @@ def lib():
         L.tngo_quot_den.argtypes = [_f32p, C.c_uint64, C.c_float, _f32p]
         L.tngo_encode.argtypes = [_f32p, C.c_int, C.c_uint64, C.c_uint64, _f32p, C.c_int, C.c_float, C.c_int,
                                   C.c_uint64, C.c_int, C.c_int, C.c_uint32, C.c_uint32, C.c_uint32, _u32p, _f32p]
-        L.tngo_encode_at.argtypes = [_f32p, C.c_int, C.c_uint64, C.c_uint64, _f32p, _f32p, C.c_int, C.c_float, C.c_int,
+        L.tngo_encode_at.argtypes = [_f32p, C.c_int, C.c_uint64, C.c_uint64, _f32p, _f32p, _f32p, C.c_int, C.c_float, C.c_int,
                                      C.c_uint64, C.c_int, C.c_int, C.c_uint32, C.c_uint32, C.c_uint32, C.c_uint64, _u32p, _f32p]
         L.tngo_decode_aggregate.argtypes = [_u32p, _f32p, C.c_int, C.c_uint64, _f32p, C.c_int, C.c_float, C.c_int,
                                             C.c_uint64, C.c_int, _f32p]
-        L.tngo_decode_aggregate2.argtypes = [_u32p, _f32p, C.c_int, C.c_uint64, _f32p, _f32p, C.c_int, C.c_float, C.c_int,
+        L.tngo_decode_aggregate2.argtypes = [_u32p, _f32p, C.c_int, C.c_uint64, _f32p, _f32p, _f32p, C.c_int, C.c_float, C.c_int,
                                              C.c_uint64, C.c_int, _f32p]
         L.tngo_magnitude_reference.argtypes = [C.POINTER(_f32p), C.c_int, C.c_uint64, _f32p]
+        L.tngo_row_mean.argtypes = [_f32p, C.c_uint64]
+        L.tngo_row_mean.restype = C.c_float
+        L.tngo_mean_of_means.argtypes = [_f32p, C.c_int]
+        L.tngo_mean_of_means.restype = C.c_float
         L.tngo_dequant.restype = C.c_float
         L.tngo_dequant.argtypes = [C.c_int, C.c_int, C.c_uint32, C.c_float]
         L.tngo_cnz.restype = C.c_double
@@ -93,7 +97,7 @@ def lib():
         L.tngo_stage_encode.argtypes = [C.c_void_p, _f32p, C.c_uint64]
         L.tngo_stage_decode_push.argtypes = [C.c_void_p, _f32p]
         for name, rt in (("tngo_ref", _f32p), ("tngo_ref2", _f32p), ("tngo_codes", _u32p), ("tngo_scales", _f32p),
-                         ("tngo_alpha", _f32p), ("tngo_gram", _f64p)):
+                         ("tngo_means", _f32p), ("tngo_alpha", _f32p), ("tngo_gram", _f64p)):
             getattr(L, name).restype = rt
             getattr(L, name).argtypes = [C.c_void_p]
         L.tngo_history.restype = _f32p
@@ -223,28 +227,48 @@ def quot_den(ref, quot_eps=2.0 ** -4):
 
 
 def encode(grads, ref, norm, codec, B=128, s=7, scale_kind=SCALE_ABSMAX, seed=(0, 0), t=0, quot_eps=2.0 ** -4,
-           coord_offset=0, ref2=None):
+           coord_offset=0, ref2=None, means=None):
     """Returns (codes[M, words_per_worker] uint32, scales[M, num_blocks] float32).  With
-    coord_offset = i0 the columns handed in are coordinates i0.. of a longer vector."""
+    coord_offset = i0 the columns handed in are coordinates i0.. of a longer vector.
+    NORM_MEAN: `means` are the workers' scalar references (row_means of the whole vectors);
+    left out, they are taken from the rows handed in."""
     g, M, ld = _rows(grads)
     d = g.shape[1]
     r = None if ref is None else np.ascontiguousarray(ref, dtype=np.float32)
     r2 = None if ref2 is None else np.ascontiguousarray(ref2, dtype=np.float32)
+    mu = None
+    if norm == NORM_MEAN:
+        mu = row_means(g) if means is None else np.ascontiguousarray(means, dtype=np.float32)
+        assert mu.shape == (M,)
     codes = np.zeros((M, words_per_worker(d, codec)), dtype=np.uint32)
     scales = np.zeros((M, num_blocks(d, B)), dtype=np.float32)
-    lib().tngo_encode_at(_ptr_f32(g), M, ld, d, _ptr_f32(r), _ptr_f32(r2), norm, quot_eps, codec, B, s, scale_kind,
+    lib().tngo_encode_at(_ptr_f32(g), M, ld, d, _ptr_f32(r), _ptr_f32(r2), _ptr_f32(mu), norm, quot_eps, codec, B, s, scale_kind,
                          seed[0], seed[1], t, int(coord_offset), codes.ctypes.data_as(_u32p), _ptr_f32(scales))
     return codes, scales
 
 
-def decode_aggregate(codes, scales, d, ref, norm, codec, B=128, s=7, quot_eps=2.0 ** -4, ref2=None):
+def row_means(grads):
+    """mean(g^m) of every row: the scalar references of NORM_MEAN (Section 3.1)."""
+    g, M, ld = _rows(grads)
+    d = g.shape[1]
+    return np.array([lib().tngo_row_mean(_ptr_f32(g[m]), d) for m in range(M)], dtype=np.float32)
+
+
+def mean_of_means(means):
+    mu = np.ascontiguousarray(means, dtype=np.float32)
+    return np.float32(lib().tngo_mean_of_means(_ptr_f32(mu), mu.shape[0]))
+
+
+def decode_aggregate(codes, scales, d, ref, norm, codec, B=128, s=7, quot_eps=2.0 ** -4, ref2=None, means=None):
     codes = np.ascontiguousarray(codes, dtype=np.uint32)
     scales = np.ascontiguousarray(scales, dtype=np.float32)
     M = codes.shape[0]
     r = None if ref is None else np.ascontiguousarray(ref, dtype=np.float32)
     r2 = None if ref2 is None else np.ascontiguousarray(ref2, dtype=np.float32)
+    mu = None if means is None else np.ascontiguousarray(means, dtype=np.float32)
+    assert norm != NORM_MEAN or (mu is not None and mu.shape == (M,))
     out = np.zeros(d, dtype=np.float32)
-    lib().tngo_decode_aggregate2(codes.ctypes.data_as(_u32p), _ptr_f32(scales), M, d, _ptr_f32(r), _ptr_f32(r2), norm,
+    lib().tngo_decode_aggregate2(codes.ctypes.data_as(_u32p), _ptr_f32(scales), M, d, _ptr_f32(r), _ptr_f32(r2), _ptr_f32(mu), norm,
                                  quot_eps, codec, B, s, _ptr_f32(out))
     return out
 
@@ -340,6 +364,9 @@ class State:
 
     def ref2(self):
         return np.ctypeslib.as_array(lib().tngo_ref2(self._h), shape=(self.d,)).copy()
+
+    def means(self):
+        return np.ctypeslib.as_array(lib().tngo_means(self._h), shape=(self.M,)).copy()
 
     def codes(self):
         w = words_per_worker(self.d, self.codec)

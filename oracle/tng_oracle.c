@@ -306,6 +306,26 @@ static float l2_scale(const float* v, uint64_t n) {
 
 static int scale_is_bad(float R) { return !(R > 0.0f) || !isfinite(R); }
 
+/* Scalar reference of Section 3.1 (fourth entry of the list of references): mean(g), the
+ * average of all elements of one worker's gradient.  The sum is the fp32 adjacent-pairwise
+ * tree over the d coordinates, zero-padded to a power of two; one IEEE division by d. */
+float tngo_row_mean(const float* g, uint64_t d) {
+    uint64_t P = pow2_ceil(d);
+    float* buf = (float*)calloc(P ? P : 1, sizeof(float));
+    for (uint64_t i = 0; i < d; ++i) buf[i] = g[i];
+    for (uint64_t len = P; len > 1; len /= 2)
+        for (uint64_t i = 0; i < len / 2; ++i) buf[i] = buf[2 * i] + buf[2 * i + 1];
+    float S = buf[0];
+    free(buf);
+    return S / (float)d;
+}
+/* What the server adds back: the average of the workers' means, summed m ascending in fp32. */
+float tngo_mean_of_means(const float* means, int M) {
+    float acc = 0.0f;
+    for (int m = 0; m < M; ++m) acc = (m == 0) ? means[m] : acc + means[m];
+    return acc / (float)M;
+}
+
 /* ------------------------------------------------------------------------- */
 /* quantisers: symbol of one coordinate given v, its block scale R and u       */
 /* ------------------------------------------------------------------------- */
@@ -356,8 +376,8 @@ float tngo_dequant(int codec, int s, uint32_t symbol, float R) {
 /* The d coordinates handed in are coordinates i0 .. i0+d-1 of a longer vector (i0 a
  * multiple of the block size and of 128): only the Philox counters see i0. */
 void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, const float* ref2,
-                    int norm, float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
-                    uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales) {
+                    const float* means, int norm, float quot_eps, int codec, uint64_t B, int s, int scale_kind,
+                    uint32_t seed_lo, uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales) {
     uint64_t wpw = tngo_words_per_worker(d, codec);
     uint64_t nblk = tngo_num_blocks(d, B);
     uint64_t Beff = (B == 0) ? d : B;
@@ -381,9 +401,11 @@ void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const fl
         uint64_t n = hi - lo;
         const float* g = grads + (uint64_t)m * ld;
         float* v = (float*)malloc(sizeof(float) * (n ? n : 1));
-        for (uint64_t i = 0; i < n; ++i)
-            v[i] = (norm == TNGO_NORM_COMB) ? normalise_comb(g[lo + i], ref ? ref[lo + i] : 0.0f, opnd[lo + i])
-                                            : normalise(g[lo + i], norm, opnd[lo + i]);
+        for (uint64_t i = 0; i < n; ++i) {
+            if (norm == TNGO_NORM_COMB) v[i] = normalise_comb(g[lo + i], ref ? ref[lo + i] : 0.0f, opnd[lo + i]);
+            else if (norm == TNGO_NORM_MEAN) v[i] = g[lo + i] - means[m];   /* reference mean(g^m) ones(D) */
+            else v[i] = normalise(g[lo + i], norm, opnd[lo + i]);
+        }
         float R = (scale_kind == TNGO_SCALE_L2) ? l2_scale(v, n) : absmax_nan(v, n);
         scales[(uint64_t)m * nblk + blk] = R;
         if (!scale_is_bad(R)) {
@@ -406,15 +428,16 @@ void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const fl
 void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, int norm,
                  float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
                  uint32_t seed_hi, uint32_t t, uint32_t* codes, float* scales) {
-    tngo_encode_at(grads, M, ld, d, ref, NULL, norm, quot_eps, codec, B, s, scale_kind, seed_lo, seed_hi, t, 0, codes, scales);
+    tngo_encode_at(grads, M, ld, d, ref, NULL, NULL, norm, quot_eps, codec, B, s, scale_kind, seed_lo, seed_hi, t, 0, codes,
+                   scales);
 }
 
 /* ------------------------------------------------------------------------- */
 /* decode + aggregate + de-normalise                                          */
 /* ------------------------------------------------------------------------- */
 void tngo_decode_aggregate2(const uint32_t* codes, const float* scales, int M, uint64_t d,
-                            const float* ref, const float* ref2, int norm, float quot_eps, int codec,
-                            uint64_t B, int s, float* out) {
+                            const float* ref, const float* ref2, const float* means, int norm, float quot_eps,
+                            int codec, uint64_t B, int s, float* out) {
     uint64_t wpw = tngo_words_per_worker(d, codec);
     uint64_t nblk = tngo_num_blocks(d, B);
     uint64_t Beff = (B == 0) ? d : B;
@@ -423,6 +446,7 @@ void tngo_decode_aggregate2(const uint32_t* codes, const float* scales, int M, u
         den = (float*)malloc(sizeof(float) * (d ? d : 1));
         tngo_quot_den(norm == TNGO_NORM_QUOT ? ref : ref2, d, quot_eps, den);
     }
+    float mbar = (norm == TNGO_NORM_MEAN) ? tngo_mean_of_means(means, M) : 0.0f;
 #pragma omp parallel for
     for (uint64_t i = 0; i < d; ++i) {
         uint64_t blk = (Beff == 0) ? 0 : i / Beff;
@@ -441,7 +465,8 @@ void tngo_decode_aggregate2(const uint32_t* codes, const float* scales, int M, u
         else if (norm == TNGO_NORM_COMB) {                    /* v = ref' . r(w_t) + ref */
             float scaled = den[i] * a;
             out[i] = scaled + r;
-        } else out[i] = a;
+        } else if (norm == TNGO_NORM_MEAN) out[i] = a + mbar; /* (1/M) sum_m (vhat^m + mean^m ones) */
+        else out[i] = a;
     }
     free(den);
 }
@@ -449,7 +474,7 @@ void tngo_decode_aggregate2(const uint32_t* codes, const float* scales, int M, u
 void tngo_decode_aggregate(const uint32_t* codes, const float* scales, int M, uint64_t d,
                            const float* ref, int norm, float quot_eps, int codec, uint64_t B,
                            int s, float* out) {
-    tngo_decode_aggregate2(codes, scales, M, d, ref, NULL, norm, quot_eps, codec, B, s, out);
+    tngo_decode_aggregate2(codes, scales, M, d, ref, NULL, NULL, norm, quot_eps, codec, B, s, out);
 }
 
 /* ------------------------------------------------------------------------- */
@@ -492,6 +517,7 @@ struct tngo_state {
     float* ref2; /* second reference (combined form) */
     uint32_t* codes;
     float* scales;
+    float means[64]; /* scalar references of the round (TNGO_NORM_MEAN) */
     double gram[TNGO_MAX_K * TNGO_MAX_K + TNGO_MAX_K + 1];
     double alpha64[TNGO_MAX_K];
     float alpha[TNGO_MAX_K];
@@ -501,7 +527,7 @@ struct tngo_state {
 tngo_state* tngo_create(uint64_t d, int M, int K, int codec, int norm) {
     if (d == 0 || M < 1 || M > 64 || K < 1 || K > TNGO_MAX_K) return NULL;
     if (codec != 1 && codec != 2 && codec != 4) return NULL;
-    if (norm < 0 || norm > 3) return NULL;
+    if (norm < 0 || norm > 4) return NULL;
     tngo_state* st = (tngo_state*)calloc(1, sizeof *st);
     st->d = d; st->M = M; st->K = K; st->codec = codec; st->norm = norm;
     st->B = 128; st->s = 7; st->scale_kind = TNGO_SCALE_ABSMAX; st->fuse_mode = 0;
@@ -599,13 +625,15 @@ void tngo_stage_fuse(tngo_state* st, const float* grads, uint64_t ld) {
 void tngo_stage_encode(tngo_state* st, const float* grads, uint64_t ld) {
     uint64_t nblk = tngo_num_blocks(st->d, st->B);
     if (!st->scales) st->scales = (float*)calloc((size_t)st->M * nblk, sizeof(float));
-    tngo_encode_at(grads, st->M, ld, st->d, st->ref, st->ref2, st->norm, st->quot_eps, st->codec, st->B, st->s,
-                   st->scale_kind, st->seed_lo, st->seed_hi, st->t, 0, st->codes, st->scales);
+    if (st->norm == TNGO_NORM_MEAN)
+        for (int m = 0; m < st->M; ++m) st->means[m] = tngo_row_mean(grads + (uint64_t)m * ld, st->d);
+    tngo_encode_at(grads, st->M, ld, st->d, st->ref, st->ref2, st->means, st->norm, st->quot_eps, st->codec, st->B,
+                   st->s, st->scale_kind, st->seed_lo, st->seed_hi, st->t, 0, st->codes, st->scales);
 }
 
 void tngo_stage_decode_push(tngo_state* st, float* out) {
-    tngo_decode_aggregate2(st->codes, st->scales, st->M, st->d, st->ref, st->ref2, st->norm, st->quot_eps,
-                           st->codec, st->B, st->s, out);
+    tngo_decode_aggregate2(st->codes, st->scales, st->M, st->d, st->ref, st->ref2, st->means, st->norm,
+                           st->quot_eps, st->codec, st->B, st->s, out);
     push(st, out);
     st->t += 1;
 }
@@ -613,7 +641,8 @@ void tngo_stage_decode_push(tngo_state* st, float* out) {
 /* Reference refresh cadence (Sec. 3.1, last paragraph): a new reference only in rounds t with
  * t % ref_every == 0; in between the previous one is kept.  The ring receives every aggregate. */
 void tngo_step(tngo_state* st, const float* grads, uint64_t ld, float* out) {
-    if (st->t % st->ref_every == 0) tngo_stage_fuse(st, grads, ld);
+    /* the scalar reference uses no trajectory */
+    if (st->norm != TNGO_NORM_MEAN && st->t % st->ref_every == 0) tngo_stage_fuse(st, grads, ld);
     tngo_stage_encode(st, grads, ld);
     tngo_stage_decode_push(st, out);
 }
@@ -622,6 +651,7 @@ const float* tngo_ref(const tngo_state* st) { return st->ref; }
 const float* tngo_ref2(const tngo_state* st) { return st->ref2; }
 const uint32_t* tngo_codes(const tngo_state* st) { return st->codes; }
 const float* tngo_scales(const tngo_state* st) { return st->scales; }
+const float* tngo_means(const tngo_state* st) { return st->means; }
 const float* tngo_alpha(const tngo_state* st) { return st->alpha; }
 const double* tngo_gram(const tngo_state* st) { return st->gram; }
 int tngo_hist_count(const tngo_state* st) { return st->k; }

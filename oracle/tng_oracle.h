@@ -29,7 +29,9 @@ extern "C" {
 
 /* codec value = bits per symbol */
 enum { TNGO_CODEC_SIGN1 = 1, TNGO_CODEC_TERN2 = 2, TNGO_CODEC_QSGD4 = 4 };
-enum { TNGO_NORM_NONE = 0, TNGO_NORM_DIFF = 1, TNGO_NORM_QUOT = 2, TNGO_NORM_COMB = 3 };
+/* MEAN: the reference of worker m is the scalar mean(g^m) times ones(D) (Section 3.1); it
+ * needs no trajectory, each worker sends its scalar along with the codes. */
+enum { TNGO_NORM_NONE = 0, TNGO_NORM_DIFF = 1, TNGO_NORM_QUOT = 2, TNGO_NORM_COMB = 3, TNGO_NORM_MEAN = 4 };
 enum { TNGO_SCALE_ABSMAX = 0, TNGO_SCALE_L2 = 1 };
 enum { TNGO_FUSE_LAST = 1, TNGO_FUSE_MEAN = 2, TNGO_FUSE_LSQ = 3, TNGO_FUSE_HINDSIGHT = 4 };
 
@@ -83,9 +85,16 @@ void tngo_encode(const float* grads, int M, uint64_t ld, uint64_t d, const float
  * multiple of 128 and of B), which only moves the Philox counters. */
 /* ref2: second reference of the combined form r = Q[(g - ref) ./ ref2], v = ref2 . r + ref
  * (Section 3, display after Eq. 3); only read when norm == TNGO_NORM_COMB. */
+/* means: the M scalar references mean(g^m) of TNGO_NORM_MEAN (of the WHOLE vectors, when the
+ * d coordinates are a window); only read in that mode. */
 void tngo_encode_at(const float* grads, int M, uint64_t ld, uint64_t d, const float* ref, const float* ref2,
-                    int norm, float quot_eps, int codec, uint64_t B, int s, int scale_kind, uint32_t seed_lo,
-                    uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales);
+                    const float* means, int norm, float quot_eps, int codec, uint64_t B, int s, int scale_kind,
+                    uint32_t seed_lo, uint32_t seed_hi, uint32_t t, uint64_t i0, uint32_t* codes, float* scales);
+/* mean(g): fp32 adjacent-pairwise tree sum over the d elements (zero-padded to a power of
+ * two) divided by d (Section 3.1, the scalar reference). */
+float tngo_row_mean(const float* g, uint64_t d);
+/* (1/M) sum_m means[m], m ascending in fp32: what decoding adds back in TNGO_NORM_MEAN. */
+float tngo_mean_of_means(const float* means, int M);
 /* r'_d = (1/k) sum_j |h_j,d|: per-coordinate magnitude of the trajectory (fp32 fma chain). */
 void tngo_magnitude_reference(const float* const* h, int k, uint64_t d, float* ref2);
 
@@ -94,8 +103,8 @@ void tngo_decode_aggregate(const uint32_t* codes, const float* scales, int M, ui
                            const float* ref, int norm, float quot_eps, int codec, uint64_t B,
                            int s, float* out);
 void tngo_decode_aggregate2(const uint32_t* codes, const float* scales, int M, uint64_t d,
-                            const float* ref, const float* ref2, int norm, float quot_eps, int codec,
-                            uint64_t B, int s, float* out);
+                            const float* ref, const float* ref2, const float* means, int norm, float quot_eps,
+                            int codec, uint64_t B, int s, float* out);
 /* Decoded value of one symbol (used by tests that unpack the wire themselves). */
 float tngo_dequant(int codec, int s, uint32_t symbol, float R);
 
@@ -123,6 +132,7 @@ const float* tngo_ref(const tngo_state* st);
 const float* tngo_ref2(const tngo_state* st);
 const uint32_t* tngo_codes(const tngo_state* st);
 const float* tngo_scales(const tngo_state* st);
+const float* tngo_means(const tngo_state* st); /* M scalar references of the last round (TNGO_NORM_MEAN) */
 const float* tngo_alpha(const tngo_state* st);
 const double* tngo_gram(const tngo_state* st); /* k*k then c (k) then gg (1) */
 int tngo_hist_count(const tngo_state* st);
