@@ -39,28 +39,35 @@ WORKLOADS = {
 }
 
 
-def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True, ref_in_encode=True):
+def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True, ref_in_encode=True, norm="quot"):
     """Bytes per coordinate each kernel of one round has to move (reads + writes).
 
     dots    reads the K ring rows and the M gradient rows;
     encode  reads the M gradient rows and writes the wire (codes + scales); with the reference
             combine folded into it (block 128) it also reads the K ring rows and writes the
             reference, otherwise it reads the reference a separate combine pass wrote;
-    decode  reads the wire and the reference, writes the new ring entry (and the caller's copy)."""
+    decode  reads the wire and the reference, writes the new ring entry (and the caller's copy).
+    The combined form carries a second reference wherever the first one is read or written; the
+    scalar reference has no fusion at all, its encode reads the gradient rows twice (means, then codes)."""
     wire = M * bits / 8.0 + 4.0 * M / block
     per = {}
+    if norm == "mean":
+        per["encode"] = 8.0 * M + wire
+        per["decode"] = wire + 4.0 + (4.0 if user_out else 0.0)
+        return per
+    refs = 8.0 if norm == "comb" else 4.0
     if fuse == "lsq":
         per["dots"] = 4.0 * K + 4.0 * M
     elif fuse == "hindsight":
         per["dots"] = 4.0 * K                      # Gram of the ring only
     combines = fuse != "last"                      # the delayed-gradient reference is a ring slot as it is
     if combines and ref_in_encode:
-        per["encode"] = 4.0 * K + 4.0 * M + 4.0 + wire
+        per["encode"] = 4.0 * K + 4.0 * M + refs + wire
     else:
         if combines:
-            per["combine"] = 4.0 * K + 4.0
-        per["encode"] = 4.0 * M + 4.0 + wire
-    per["decode"] = wire + 4.0 + 4.0 + (4.0 if user_out else 0.0)
+            per["combine"] = 4.0 * K + refs
+        per["encode"] = 4.0 * M + refs + wire
+    per["decode"] = wire + refs + 4.0 + (4.0 if user_out else 0.0)
     return per
 
 
@@ -132,7 +139,8 @@ class ClockSampler(threading.Thread):
 
 
 def enum_of(tng, cfg):
-    norm = {"none": tng.NORM_NONE, "diff": tng.NORM_DIFF, "quot": tng.NORM_QUOT}[cfg["norm"]]
+    norm = {"none": tng.NORM_NONE, "diff": tng.NORM_DIFF, "quot": tng.NORM_QUOT, "comb": tng.NORM_COMB,
+            "mean": tng.NORM_MEAN}[cfg["norm"]]
     codec = {"sign1": tng.CODEC_SIGN1, "tern2": tng.CODEC_TERN2, "qsgd4": tng.CODEC_QSGD4}[cfg["codec"]]
     fuse = {"lsq": tng.FUSE_LSQ, "last": tng.FUSE_LAST, "mean": tng.FUSE_MEAN, "hindsight": tng.FUSE_HINDSIGHT}[cfg["fuse"]]
     return norm, codec, fuse
@@ -292,8 +300,8 @@ def run_ours(args, name, cfg):
     n0, n1 = st0.timed_rounds, st1.timed_rounds
     def stage_ms(field):
         return (getattr(st1, field) * n1 - getattr(st0, field) * n0) / max(n1 - n0, 1)
-    ref_in_encode = cfg["block"] == 128 and cfg["norm"] != "none" and stage_ms("ms_combine") == 0.0
-    per_coord = algorithmic_bytes_per_coord(M, K, bits, cfg["block"], cfg["fuse"], ref_in_encode=ref_in_encode)
+    ref_in_encode = cfg["block"] == 128 and cfg["norm"] not in ("none", "mean") and stage_ms("ms_combine") == 0.0
+    per_coord = algorithmic_bytes_per_coord(M, K, bits, cfg["block"], cfg["fuse"], ref_in_encode=ref_in_encode, norm=cfg["norm"])
     peak, peak_src = measured_hbm_peak()
     kernels = {}
     for kname, field in (("dots", "ms_dots"), ("combine", "ms_combine"), ("encode", "ms_encode"), ("decode", "ms_decode")):
@@ -306,7 +314,9 @@ def run_ours(args, name, cfg):
         kernels["encode"]["includes"] = "reference combine (ring rows -> reference) folded into the encode pass"
     kernels["solve"] = {"ms": stage_ms("ms_solve")}
     dominant = max((k for k in kernels if "bytes_per_coord" in kernels[k]), key=lambda k: kernels[k]["ms"])
-    tpc = NCU_TRAFFIC_BYTES_PER_COORD.get(dominant)
+    # the counters were taken on the headline configuration; any other one has no capture
+    profiled = all(cfg[k] == WORKLOADS["c5_dnn_stream"][k] for k in ("M", "K", "norm", "codec", "block", "fuse"))
+    tpc = NCU_TRAFFIC_BYTES_PER_COORD.get(dominant) if profiled else None
     traffic = tpc * d if tpc is not None else None
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["GBps"], "peak": peak, "unit": "GB/s",
                 "frac": kernels[dominant]["frac_of_measured"], "peak_source": peak_src, "traffic": traffic,
@@ -421,7 +431,7 @@ def main():
     # overrides for sweeps over the codec-sweep configuration (not the headline line)
     ap.add_argument("--d", type=int, default=None)
     ap.add_argument("--codec", choices=["sign1", "tern2", "qsgd4"], default=None)
-    ap.add_argument("--norm", choices=["none", "diff", "quot"], default=None)
+    ap.add_argument("--norm", choices=["none", "diff", "quot", "comb", "mean"], default=None)
     ap.add_argument("--fuse", choices=["lsq", "last", "mean", "hindsight"], default=None)
     args = ap.parse_args()
     if args.workload == "producers":

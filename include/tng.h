@@ -50,8 +50,13 @@ typedef enum {
 typedef enum { TNG_CODEC_SIGN1 = 1, TNG_CODEC_TERN2 = 2, TNG_CODEC_QSGD4 = 4 } tng_codec;
 /* NONE: v = g.  DIFF: Eq. 2.  QUOT: Eq. 3.  COMB: the combined form of Section 3,
  * r = Q[(g - ref) ./ ref'], v = ref' . r + ref, with ref' = the mean absolute value of the
- * stored aggregates (per coordinate), guarded like the quotient form's denominator. */
-typedef enum { TNG_NORM_NONE = 0, TNG_NORM_DIFF = 1, TNG_NORM_QUOT = 2, TNG_NORM_COMB = 3 } tng_norm_mode;
+ * stored aggregates (per coordinate), guarded like the quotient form's denominator.
+ * MEAN: the scalar reference of Section 3.1, ref^m = mean(g^m) ones(D): v = g^m - mean(g^m),
+ * every worker sends its scalar along with codes and scales (tng_wire_means), decoding adds
+ * the average of the M scalars back.  mean(g) is the fp32 adjacent-pairwise tree sum of the
+ * d elements divided by d.  No trajectory is used: the fusion stage is skipped (the ring
+ * still receives every aggregate). */
+typedef enum { TNG_NORM_NONE = 0, TNG_NORM_DIFF = 1, TNG_NORM_QUOT = 2, TNG_NORM_COMB = 3, TNG_NORM_MEAN = 4 } tng_norm_mode;
 typedef enum {
     TNG_FUSE_AUTO = 0,     /* K == 1 -> LAST, else LSQ */
     TNG_FUSE_LAST = 1,     /* r = newest aggregate (delayed gradient, Sec. 3.1 / Sec. 4.2 protocol) */
@@ -208,6 +213,9 @@ tng_status tng_decode_commit(tng_ctx* ctx, float* agg_out_dev, void* stream);
  * is bit p of the symbol of coordinate 128T + 4j + c. */
 tng_status tng_wire(tng_ctx* ctx, const uint32_t** codes_dev, size_t* words_per_worker,
                     const float** scales_dev, size_t* scales_per_worker);
+/* TNG_NORM_MEAN: the M scalars mean(g^m) of the last encode (device, M floats; part of the
+ * wire: with the workers on different GPUs they are gathered like the scales). */
+tng_status tng_wire_means(tng_ctx* ctx, const float** means_dev);
 tng_status tng_reference(tng_ctx* ctx, const float** ref_dev);
 /* h_{j+1}: j = 0 is the newest stored aggregate; j < k. */
 tng_status tng_history(tng_ctx* ctx, uint32_t j, const float** vec_dev);

@@ -40,7 +40,7 @@ struct tng_ctx {
     size_t ws_bytes = 0;
     bool ws_owned = false, ws_ready = false;
     size_t off_ring = 0, off_ref = 0, off_codes = 0, off_scales = 0, off_tile_stat = 0, off_tree = 0,
-           off_partials = 0, off_fb = 0, off_stage_g = 0, off_stage_o = 0, off_ref2 = 0;
+           off_partials = 0, off_fb = 0, off_stage_g = 0, off_stage_o = 0, off_ref2 = 0, off_means = 0;
     // state
     uint32_t k = 0;
     int head = 0;
@@ -69,6 +69,9 @@ struct tng_ctx {
     float* ref2_buf() const { return norm == TNG_NORM_COMB ? reinterpret_cast<float*>(static_cast<char*>(ws) + off_ref2) : nullptr; }
     uint32_t* codes() const { return reinterpret_cast<uint32_t*>(static_cast<char*>(ws) + off_codes); }
     float* scales() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_scales); }
+    float* means() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_means); }
+    // no trajectory reference is involved: plain compression or the scalar reference of Section 3.1
+    bool no_ref() const { return norm == TNG_NORM_NONE || norm == TNG_NORM_MEAN; }
     float* tile_stat() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_tile_stat); }
     float* tree() const { return reinterpret_cast<float*>(static_cast<char*>(ws) + off_tree); }
     double* partials() const { return reinterpret_cast<double*>(static_cast<char*>(ws) + off_partials); }
@@ -114,8 +117,8 @@ void size_ctx(tng_ctx* c) {
     c->off_ref2 = off;      off += align_up(c->norm == TNG_NORM_COMB ? (size_t)c->d_pad * sizeof(float) : 0);
     c->off_codes = off;     off += align_up((size_t)c->M * g.wpw * sizeof(uint32_t));
     c->off_scales = off;    off += align_up((size_t)c->M * g.nblk * sizeof(float));
-    const bool general = g.block != TNG_TILE;
-    c->off_tile_stat = off; off += align_up(general ? (size_t)c->M * g.ntile * sizeof(float) : 0);
+    c->off_means = off;     off += align_up((size_t)TNG_MAX_WORKERS * sizeof(float));
+    c->off_tile_stat = off; off += align_up(encode_needs_tile_stat(g) ? (size_t)c->M * g.ntile * sizeof(float) : 0);
     c->off_tree = off;      off += align_up(tree_tmp_floats(g) * sizeof(float));
     c->off_partials = off;  off += align_up((size_t)kDotsMaxCtas * kDotsMaxAcc * sizeof(double));
     c->off_fb = off;        off += align_up(sizeof(FuseBlock));
@@ -253,15 +256,16 @@ tng_status do_fuse(tng_ctx* c, const float* grads, uint64_t ld, cudaStream_t st,
 tng_status do_encode(tng_ctx* c, const float* grads, uint64_t ld, const float* ref, const RefFusion* fusion, uint32_t step,
                      cudaStream_t st) {
     int launches = 0;
-    TNG_CUDA(c, launch_encode(c->geom, 0, grads, ld, ref, c->ref2_buf(), fusion, step, c->codes(), c->scales(), c->tile_stat(), c->tree(),
-                              c->fb(), c->sm_count, st, &launches));
+    TNG_CUDA(c, launch_encode(c->geom, 0, grads, ld, ref, c->ref2_buf(), fusion, step, c->codes(), c->scales(), c->means(),
+                              c->tile_stat(), c->tree(), c->fb(), c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
 }
 
 tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, cudaStream_t st) {
     int launches = 0;
-    TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), ref, c->ref2_buf(), out_a, out_b, c->fb(), c->sm_count, st, &launches));
+    TNG_CUDA(c, launch_decode(c->geom, c->codes(), c->scales(), c->means(), ref, c->ref2_buf(), out_a, out_b, c->fb(), c->sm_count, st,
+                              &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
 }
@@ -283,7 +287,9 @@ tng_status step_impl(tng_ctx* c, const float* grads, uint64_t ld, float* out, cu
     RefFusion fusion;
     fusion.k = 0;
     tng_status s = TNG_OK;
-    if (c->rounds % c->ref_every == 0 || !c->ref_cur) {
+    if (c->norm == TNG_NORM_MEAN) {   // the scalar reference uses no trajectory
+        tm.mark(0, false); tm.mark(1, false); tm.mark(2, false);
+    } else if (c->rounds % c->ref_every == 0 || !c->ref_cur) {
         s = do_fuse(c, grads, ld, st, &tm, &fusion);
         if (s != TNG_OK) return s;
         if (c->ref_every > 1 && c->ref_cur != c->ref_buf()) {
@@ -313,7 +319,8 @@ tng_status tng_create(tng_ctx** out, uint64_t d, uint32_t M, uint32_t K, tng_cod
     *out = nullptr;
     if (d < 1 || d > TNG_MAX_COORDS || M < 1 || M > TNG_MAX_WORKERS || K < 1 || K > TNG_MAX_HISTORY) return TNG_ERR_INVALID_ARG;
     if (codec != TNG_CODEC_SIGN1 && codec != TNG_CODEC_TERN2 && codec != TNG_CODEC_QSGD4) return TNG_ERR_INVALID_ARG;
-    if (norm != TNG_NORM_NONE && norm != TNG_NORM_DIFF && norm != TNG_NORM_QUOT && norm != TNG_NORM_COMB) return TNG_ERR_INVALID_ARG;
+    if (norm != TNG_NORM_NONE && norm != TNG_NORM_DIFF && norm != TNG_NORM_QUOT && norm != TNG_NORM_COMB && norm != TNG_NORM_MEAN)
+        return TNG_ERR_INVALID_ARG;
     tng_ctx* c = new (std::nothrow) tng_ctx();
     if (!c) return TNG_ERR_ALLOC;
     c->d = d; c->M = M; c->K = K; c->codec = (int)codec; c->norm = (int)norm;
@@ -563,13 +570,14 @@ tng_status tng_encode_local(tng_ctx* c, const float* grads_dev, uint64_t ld, uin
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
-    if (!c->ref_cur && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;   // no fusion has produced a reference yet
+    if (!c->ref_cur && !c->no_ref()) return TNG_ERR_STATE;   // no fusion has produced a reference yet
     if (c->norm == TNG_NORM_COMB && !c->ref2_valid) return TNG_ERR_STATE;
     CodecGeom g = c->geom;
     g.M = m_count;
     int launches = 0;
     TNG_CUDA(c, launch_encode(g, m_first, grads_dev, ld, c->ref_cur, c->ref2_buf(), nullptr, step, c->codes() + (size_t)m_first * g.wpw,
-                              c->scales() + (size_t)m_first * g.nblk, c->tile_stat(), c->tree(), c->fb(), c->sm_count, st, &launches));
+                              c->scales() + (size_t)m_first * g.nblk, c->means() + m_first, c->tile_stat(), c->tree(), c->fb(),
+                              c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
     return TNG_OK;
 }
@@ -580,7 +588,7 @@ tng_status tng_decode_commit(tng_ctx* c, float* agg_out_dev, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     tng_status s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
-    if (!c->ref_cur && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;
+    if (!c->ref_cur && !c->no_ref()) return TNG_ERR_STATE;
     return decode_commit(c, agg_out_dev, st);
 }
 
@@ -603,7 +611,7 @@ tng_status tng_encode(tng_ctx* c, const float* grads_dev, uint64_t ld, const flo
     s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
     const float* ref = ref_dev ? ref_dev : c->ref_cur;
-    if (!ref && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;   // no fusion has produced a reference yet
+    if (!ref && !c->no_ref()) return TNG_ERR_STATE;   // no fusion has produced a reference yet
     if (c->norm == TNG_NORM_COMB && !c->ref2_valid) return TNG_ERR_STATE;   // the second reference comes from a fusion
     return do_encode(c, grads_dev, ld, ref, nullptr, step, st);
 }
@@ -615,7 +623,7 @@ tng_status tng_decode_aggregate(tng_ctx* c, const float* ref_dev, float* out_dev
     tng_status s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
     const float* ref = ref_dev ? ref_dev : c->ref_cur;
-    if (!ref && c->norm != TNG_NORM_NONE) return TNG_ERR_STATE;
+    if (!ref && !c->no_ref()) return TNG_ERR_STATE;
     if (c->norm == TNG_NORM_COMB && !c->ref2_valid) return TNG_ERR_STATE;
     return do_decode(c, ref, out_dev, nullptr, st);
 }
@@ -628,6 +636,13 @@ tng_status tng_wire(tng_ctx* c, const uint32_t** codes_dev, size_t* words_per_wo
     if (words_per_worker) *words_per_worker = (size_t)c->geom.wpw;
     if (scales_dev) *scales_dev = c->scales();
     if (scales_per_worker) *scales_per_worker = (size_t)c->geom.nblk;
+    return TNG_OK;
+}
+
+tng_status tng_wire_means(tng_ctx* c, const float** means_dev) {
+    if (!c || !means_dev) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready) return TNG_ERR_STATE;
+    *means_dev = c->means();
     return TNG_OK;
 }
 

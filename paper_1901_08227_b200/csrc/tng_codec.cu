@@ -51,6 +51,8 @@ struct EncodeArgs {
     const float* ref2;
     float* ref2_out;
     float inv_k;
+    // scalar reference (TNG_NORM_MEAN): means[m] = mean(g^m) of the launch's worker m
+    const float* means;
 };
 
 // max(|a|, |b|) that returns NaN if either is NaN
@@ -95,7 +97,7 @@ __device__ __forceinline__ void encode_normalise(const float4 g, const NormOp& o
         v[2] = __fmul_rn(__fsub_rn(g.z, op.z), opn.b.z); v[3] = __fmul_rn(__fsub_rn(g.w, op.w), opn.b.w);
         return;
     }
-    if (NORM == TNG_NORM_DIFF) {
+    if (NORM == TNG_NORM_DIFF || NORM == TNG_NORM_MEAN) {
         v[0] = __fsub_rn(g.x, op.x); v[1] = __fsub_rn(g.y, op.y); v[2] = __fsub_rn(g.z, op.z); v[3] = __fsub_rn(g.w, op.w);
     } else if (NORM == TNG_NORM_QUOT) {
         v[0] = __fmul_rn(g.x, op.x); v[1] = __fmul_rn(g.y, op.y); v[2] = __fmul_rn(g.z, op.z); v[3] = __fmul_rn(g.w, op.w);
@@ -191,7 +193,13 @@ __device__ __forceinline__ uint32_t encode_worker(const EncodeArgs& a, const flo
     float R;
     uint4 x = make_uint4(0u, 0u, 0u, 0u);
     if (PHASE != kPhaseStat) x = philox4x32_10_rk(q_lo, q_hi, a.m_base + m, a.step, a.rk);
-    if (!encode_symbols<CODEC, NORM, SCALE, PHASE, FULL>(a, g, op, m, T, x, blk, lane, valid, w, R)) return 0u;
+    NormOp opm = op;
+    if (NORM == TNG_NORM_MEAN) {   // the worker's own scalar, the same for every coordinate (Section 3.1)
+        // elements past the end of the vector read as zero and must stay zero after the subtraction
+        const float mu = __ldg(a.means + m);
+        opm.a = make_float4((valid & 1u) ? mu : 0.0f, (valid & 2u) ? mu : 0.0f, (valid & 4u) ? mu : 0.0f, (valid & 8u) ? mu : 0.0f);
+    }
+    if (!encode_symbols<CODEC, NORM, SCALE, PHASE, FULL>(a, g, opm, m, T, x, blk, lane, valid, w, R)) return 0u;
     if (lane == 0) {
         uint4* dst = reinterpret_cast<uint4*>(a.codes + ((uint64_t)m * a.wpw + T * (uint64_t)kWords));
 #pragma unroll
@@ -222,7 +230,7 @@ __device__ __forceinline__ void encode_tile(const EncodeArgs& a, const float* s_
         if ((uint32_t)k < a.M) g[k] = load_row(k);
 
     NormOp op = make_norm_op<TNG_NORM_NONE>(make_float4(0.f, 0.f, 0.f, 0.f), make_float4(0.f, 0.f, 0.f, 0.f), 0.f);
-    if (NORM != TNG_NORM_NONE) {
+    if (NORM != TNG_NORM_NONE && NORM != TNG_NORM_MEAN) {
         float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
         if (FUSEREF) {
             for (int j0 = 0; j0 < a.hist_k; j0 += 4) {
@@ -449,16 +457,39 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
     }
 }
 
+// Scalar reference (Section 3.1), first pass: the sum of every tile of every row, as the
+// adjacent-pairwise fp32 tree (the lane's four values pairwise, then xor-shuffles pair
+// neighbouring lanes); elements past the end count as zero.  The tree over the tiles and
+// the division by d follow in block_scale_level_kernel<kTreeSum>.
+__global__ void __launch_bounds__(kCodecThreads) row_tile_sum_kernel(const float* __restrict__ grads, uint32_t ld, uint32_t M,
+                                                                       uint64_t d, uint64_t ntile, float* __restrict__ tile_sum) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t nwarps = (uint64_t)gridDim.x * (kCodecThreads / 32);
+    for (uint64_t T = (uint64_t)blockIdx.x * (kCodecThreads / 32) + (threadIdx.x >> 5); T < ntile; T += nwarps) {
+        const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
+        for (uint32_t m = 0; m < M; ++m) {
+            const float4 g = load4_stream(grads + (uint64_t)m * ld, i0, d);
+            float s = __fadd_rn(__fadd_rn(g.x, g.y), __fadd_rn(g.z, g.w));
+#pragma unroll
+            for (int off = 1; off < 32; off <<= 1) s = __fadd_rn(s, __shfl_xor_sync(kFullMask, s, off));
+            if (lane == 0) tile_sum[(uint64_t)m * ntile + T] = s;
+        }
+    }
+}
+
 // One level of the per-block scale reduction.  Row m holds n_in entries split
 // into segments of `seg` entries (the last one ragged); CTA (segment, chunk)
 // reduces entries [chunk*1024, chunk*1024+1024) of its segment, zero-padded, with
 // an adjacent-pairwise tree (sum) or a NaN-propagating max, and writes one value.
 // At the last level (chunks_per_seg == 1, final = 1) the value becomes the scale.
+// SCALE 2 is the plain sum behind the scalar reference: its last level divides by `divisor`
+// (the vector length) and the value becomes the worker's mean.
+constexpr int kTreeSum = 2;
 template <int SCALE>
 __global__ void __launch_bounds__(256) block_scale_level_kernel(const float* __restrict__ in, uint64_t n_in,
                                                                 uint64_t seg, uint64_t chunks_per_seg,
                                                                 float* __restrict__ out, uint64_t n_out,
-                                                                int final, unsigned long long* nonfinite) {
+                                                                int final, float divisor, unsigned long long* nonfinite) {
     __shared__ float buf[1024];
     const uint64_t s = blockIdx.x, c = blockIdx.y, m = blockIdx.z;
     const uint64_t seg_lo = s * seg;
@@ -487,7 +518,8 @@ __global__ void __launch_bounds__(256) block_scale_level_kernel(const float* __r
         float r = buf[0];
         if (final) {
             if (SCALE == 1) r = __fsqrt_rn(r);
-            if (!(r < __int_as_float(0x7f800000))) atomicAdd(nonfinite, 1ull);
+            if (SCALE == kTreeSum) r = __fdiv_rn(r, divisor);
+            if (!(fabsf(r) < __int_as_float(0x7f800000))) atomicAdd(nonfinite, 1ull);
         }
         out[m * n_out + s * chunks_per_seg + c] = r;
     }
@@ -498,6 +530,7 @@ struct DecodeArgs {
     const float* scales;
     const float* ref;
     const float* ref2;     // second reference (combined form)
+    const float* means;    // the M scalar references (TNG_NORM_MEAN)
     float* out_a;
     float* out_b;
     uint32_t* pipe_error;
@@ -585,7 +618,7 @@ __device__ __forceinline__ void decode_finish(const DecodeArgs& a, const float (
         const float fm = (float)a.M;
         o.x = __fdiv_rn(acc[0], fm); o.y = __fdiv_rn(acc[1], fm); o.z = __fdiv_rn(acc[2], fm); o.w = __fdiv_rn(acc[3], fm);
     }
-    if (NORM == TNG_NORM_DIFF) {
+    if (NORM == TNG_NORM_DIFF || NORM == TNG_NORM_MEAN) {   // MEAN: r holds the average of the workers' scalars
         o.x = __fadd_rn(r.x, o.x); o.y = __fadd_rn(r.y, o.y); o.z = __fadd_rn(r.z, o.z); o.w = __fadd_rn(r.w, o.w);
     } else if (NORM == TNG_NORM_QUOT) {
         const float4 den = quot_den4(r, a.quot_eps);
@@ -697,7 +730,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
     const uint64_t nfull = a.d / kTile;
     const uint32_t pw = a.one << (31 - lane);
     const bool tiled = a.block == (uint64_t)kTile;
-    const bool has_ref = (NORM != TNG_NORM_NONE) && a.ref != nullptr;
+    const bool has_ref = (NORM != TNG_NORM_NONE) && (NORM != TNG_NORM_MEAN) && a.ref != nullptr;
     const uint32_t n0 = a.M < kRound ? a.M : kRound;                 // workers of the first round
     // the sum starts from -0 so that (-0) + x == x bit for bit; the ternary path starts from +0
     // because it skips zero symbols and +0 is what the sum of skipped terms is
@@ -707,6 +740,14 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
     uint4 cw = make_uint4(0u, 0u, 0u, 0u);
     float sc = 0.0f;
     float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
+    if (NORM == TNG_NORM_MEAN) {
+        // what every element gets back: (1/M) sum_m mean(g^m), summed m ascending like the codes
+        float sum = a.means[0];
+        for (uint32_t m = 1; m < a.M; ++m) sum = __fadd_rn(sum, a.means[m]);
+        const float mbar = (a.inv_m > 0.0f) ? __fmul_rn(sum, a.inv_m) : __fdiv_rn(sum, (float)a.M);
+        r = make_float4(mbar, mbar, mbar, mbar);
+    }
+    const float4 r_const = r;
     const bool has_ref2 = (NORM == TNG_NORM_COMB) && a.ref2 != nullptr;
     if (T < nfull) {
         decode_fetch<CODEC>(a, T, tiled ? T : (T * kTile) / a.block, 0, lane, cw, sc);
@@ -743,7 +784,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
     if (nfull < a.ntile && gwarp == nfull % nwarps) {
         const uint64_t Tr = nfull, i0 = Tr * kTile + (uint64_t)lane * 4u;
         const uint64_t blk = tiled ? Tr : (Tr * kTile) / a.block;
-        float4 rr = make_float4(0.f, 0.f, 0.f, 0.f), rr2 = rr;
+        float4 rr = (NORM == TNG_NORM_MEAN) ? r_const : make_float4(0.f, 0.f, 0.f, 0.f), rr2 = make_float4(0.f, 0.f, 0.f, 0.f);
         if (has_ref) rr = load4(a.ref, i0, a.d);
         if (has_ref2) rr2 = load4(a.ref2, i0, a.d);
         float acc[4] = {z, z, z, z};
@@ -827,13 +868,14 @@ cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t
 
 template <int CODEC, int NORM, int SCALE, int PHASE>
 cudaError_t encode_launch(const EncodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
-    if (PHASE == kPhaseFused) {
+    if constexpr (PHASE == kPhaseFused && NORM != TNG_NORM_MEAN) {   // the scalar reference takes the direct kernels
         if (NORM != TNG_NORM_NONE && a.hist_k > 0)
             return encode_launch_tiles<CODEC, NORM, SCALE, (NORM != TNG_NORM_NONE)>(a, sm_count, st, launches);
         return encode_launch_tiles<CODEC, NORM, SCALE, false>(a, sm_count, st, launches);
+    } else {
+        ++*launches;
+        return encode_launch_direct<CODEC, NORM, SCALE, PHASE, false>(a, sm_count, st);
     }
-    ++*launches;
-    return encode_launch_direct<CODEC, NORM, SCALE, PHASE, false>(a, sm_count, st);
 }
 template <int CODEC, int NORM, int SCALE>
 cudaError_t encode_dispatch_phase(const EncodeArgs& a, int phase, int sm_count, cudaStream_t st, int* launches) {
@@ -852,6 +894,7 @@ cudaError_t encode_dispatch_norm(const EncodeArgs& a, int norm, int scale, int p
         case TNG_NORM_DIFF: return encode_dispatch_scale<CODEC, TNG_NORM_DIFF>(a, scale, phase, sm_count, st, launches);
         case TNG_NORM_QUOT: return encode_dispatch_scale<CODEC, TNG_NORM_QUOT>(a, scale, phase, sm_count, st, launches);
         case TNG_NORM_COMB: return encode_dispatch_scale<CODEC, TNG_NORM_COMB>(a, scale, phase, sm_count, st, launches);
+        case TNG_NORM_MEAN: return encode_dispatch_scale<CODEC, TNG_NORM_MEAN>(a, scale, phase, sm_count, st, launches);
         default: return encode_dispatch_scale<CODEC, TNG_NORM_NONE>(a, scale, phase, sm_count, st, launches);
     }
 }
@@ -881,6 +924,7 @@ cudaError_t decode_dispatch_norm(const DecodeArgs& a, int norm, int sm_count, cu
         case TNG_NORM_DIFF: return decode_launch<CODEC, TNG_NORM_DIFF>(a, sm_count, st, launches);
         case TNG_NORM_QUOT: return decode_launch<CODEC, TNG_NORM_QUOT>(a, sm_count, st, launches);
         case TNG_NORM_COMB: return decode_launch<CODEC, TNG_NORM_COMB>(a, sm_count, st, launches);
+        case TNG_NORM_MEAN: return decode_launch<CODEC, TNG_NORM_MEAN>(a, sm_count, st, launches);
         default: return decode_launch<CODEC, TNG_NORM_NONE>(a, sm_count, st, launches);
     }
 }
@@ -888,20 +932,26 @@ cudaError_t decode_dispatch_norm(const DecodeArgs& a, int norm, int sm_count, cu
 }  // namespace
 
 size_t tree_tmp_floats(const CodecGeom& g) {
-    if (g.block == kTile) return 0;
+    // the scalar reference reduces all tiles of a row: two ping-pong levels of M * ceil(ntile / 1024)
+    const uint64_t mean_tmp = (g.norm == TNG_NORM_MEAN) ? 2 * (uint64_t)g.M * ((g.ntile + 1023) / 1024) : 0;
+    if (g.block == kTile) return (size_t)mean_tmp;
     const uint64_t seg = (g.block + kTile - 1) / kTile;            // tiles per block
     const uint64_t chunks = (seg + 1023) / 1024;
     // two ping-pong levels, each at most M * nblk * chunks entries
-    return (size_t)(2 * (uint64_t)g.M * g.nblk * chunks);
+    const uint64_t scale_tmp = 2 * (uint64_t)g.M * g.nblk * chunks;
+    return (size_t)(scale_tmp > mean_tmp ? scale_tmp : mean_tmp);
 }
 
-bool encode_can_fuse_reference(const CodecGeom& g) { return g.block == kTile && g.norm != TNG_NORM_NONE; }
+bool encode_needs_tile_stat(const CodecGeom& g) { return g.block != kTile || g.norm == TNG_NORM_MEAN; }
+
+bool encode_can_fuse_reference(const CodecGeom& g) { return g.block == kTile && g.norm != TNG_NORM_NONE && g.norm != TNG_NORM_MEAN; }
 
 cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grads, uint64_t ld, const float* ref, const float* ref2,
                           const RefFusion* fusion,
-                          uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp, FuseBlock* fb,
-                          int sm_count, cudaStream_t st, int* launches) {
+                          uint32_t step, uint32_t* codes, float* scales, float* means, float* tile_stat, float* tree_tmp,
+                          FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
     EncodeArgs a;
+    a.means = means;
     a.hist_k = 0; a.alpha = nullptr; a.ref_out = nullptr;
     a.ref2 = ref2; a.ref2_out = nullptr; a.inv_k = 0.0f;
     for (int j = 0; j < kMaxK; ++j) a.hist[j] = nullptr;
@@ -917,6 +967,31 @@ cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grad
     a.quot_eps = g.quot_eps;
     philox_round_keys(g.seed_lo, g.seed_hi, a.rk);
     cudaError_t e;
+    if (g.norm == TNG_NORM_MEAN) {
+        // scalar reference: per-tile sums of every row, then the tree over the tiles, divided by d
+        const uint64_t want = (g.ntile + 7) / 8, cap = (uint64_t)sm_count * 8u;
+        row_tile_sum_kernel<<<(unsigned)(want < cap ? want : cap), kCodecThreads, 0, st>>>(grads, (uint32_t)ld, g.M, g.d, g.ntile, tile_stat);
+        ++*launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        const float* in = tile_stat;
+        uint64_t n_in = g.ntile;
+        float* ping = tree_tmp;
+        float* pong = tree_tmp + (uint64_t)g.M * ((g.ntile + 1023) / 1024);
+        for (;;) {
+            const uint64_t chunks = (n_in + 1023) / 1024;
+            const int final = chunks == 1;
+            dim3 grid3(1u, (unsigned)chunks, g.M);
+            block_scale_level_kernel<kTreeSum><<<grid3, 256, 0, st>>>(in, n_in, n_in, chunks, final ? means : ping, chunks, final,
+                                                                      (float)g.d, &fb->nonfinite);
+            ++*launches;
+            e = cudaGetLastError();
+            if (e != cudaSuccess) return e;
+            if (final) break;
+            in = ping; n_in = chunks;
+            float* t = ping; ping = pong; pong = t;
+        }
+    }
     if (g.block == kTile) return encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseFused, sm_count, st, launches);
     // general block size: per-tile statistic -> per-block tree -> quantise
     e = encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseStat, sm_count, st, launches);
@@ -933,9 +1008,9 @@ cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grad
         const uint64_t n_out = g.nblk * chunks;
         dim3 grid3((unsigned)g.nblk, (unsigned)chunks, g.M);
         if (g.scale_kind == 0)
-            block_scale_level_kernel<0><<<grid3, 256, 0, st>>>(in, n_in, seg, chunks, out, n_out, final, &fb->nonfinite);
+            block_scale_level_kernel<0><<<grid3, 256, 0, st>>>(in, n_in, seg, chunks, out, n_out, final, 1.0f, &fb->nonfinite);
         else
-            block_scale_level_kernel<1><<<grid3, 256, 0, st>>>(in, n_in, seg, chunks, out, n_out, final, &fb->nonfinite);
+            block_scale_level_kernel<1><<<grid3, 256, 0, st>>>(in, n_in, seg, chunks, out, n_out, final, 1.0f, &fb->nonfinite);
         ++*launches;
         e = cudaGetLastError();
         if (e != cudaSuccess || final) break;
@@ -946,10 +1021,10 @@ cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grad
     return encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseQuant, sm_count, st, launches);
 }
 
-cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref, const float* ref2,
-                          float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
+cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* means, const float* ref,
+                          const float* ref2, float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches) {
     DecodeArgs a;
-    a.codes = codes; a.scales = scales; a.ref = ref; a.ref2 = ref2; a.out_a = out_a; a.out_b = out_b;
+    a.codes = codes; a.scales = scales; a.means = means; a.ref = ref; a.ref2 = ref2; a.out_a = out_a; a.out_b = out_b;
     a.pipe_error = &fb->pipe_error; a.tile_begin = 0;
     a.d = g.d; a.ntile = g.ntile; a.nblk = (uint32_t)g.nblk; a.block = g.block; a.wpw = (uint32_t)g.wpw; a.M = g.M;
     a.one = 1u; a.levels = g.levels; a.quot_eps = g.quot_eps;

@@ -57,9 +57,10 @@ cudaError_t launch_combine(const float* const* rows, int k, uint64_t d, const Fu
                            int sm_count, cudaStream_t st, int* launches);
 
 // ---- codec (tng_codec.cu) -----------------------------------------------------
-// tile_stat: M*ntile floats, tree_tmp: scratch of tree_tmp_floats(geom) floats; both
-// only used when geom.block != 128.
+// tile_stat: M*ntile floats (needed when encode_needs_tile_stat), tree_tmp: scratch of
+// tree_tmp_floats(geom) floats; used when geom.block != 128 and by the scalar reference.
 size_t tree_tmp_floats(const CodecGeom& g);
+bool encode_needs_tile_stat(const CodecGeom& g);
 // Optional: let the encode pass build the reference itself, r = sum_j alpha[j] rows[j] (the
 // combine step's fp32 fma chain), writing it to ref_out; saves one pass over the ring and
 // hides the encode arithmetic behind the ring's memory traffic.  Only for block == 128 with
@@ -73,11 +74,12 @@ struct RefFusion {
 };
 bool encode_can_fuse_reference(const CodecGeom& g);
 // The g.M rows at `grads` are workers m_base .. m_base + g.M - 1 (their Philox streams); codes and
-// scales point at the wire slot of worker m_base.
+// scales (and means, the scalar references written in TNG_NORM_MEAN) point at the wire slot of worker m_base.
 cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grads, uint64_t ld, const float* ref, const float* ref2,
-                          const RefFusion* fusion, uint32_t step, uint32_t* codes, float* scales, float* tile_stat, float* tree_tmp,
-                          FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
-cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* ref, const float* ref2,
-                          float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
+                          const RefFusion* fusion, uint32_t step, uint32_t* codes, float* scales, float* means, float* tile_stat,
+                          float* tree_tmp, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
+// means: the M scalar references (read in TNG_NORM_MEAN only)
+cudaError_t launch_decode(const CodecGeom& g, const uint32_t* codes, const float* scales, const float* means, const float* ref,
+                          const float* ref2, float* out_a, float* out_b, FuseBlock* fb, int sm_count, cudaStream_t st, int* launches);
 
 }  // namespace tng

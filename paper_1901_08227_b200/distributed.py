@@ -7,6 +7,9 @@ every server codes its gradient, the codes are exchanged, everyone decodes the s
     fuse_local -> all-reduce of 17 doubles -> fuse_finish -> encode_local
                -> all-gather of the wire (codes and scales) -> decode_commit
 
+(with the scalar reference of Section 3.1 the fusion stages drop out and the workers' scalars
+are gathered with the wire).
+
 Only plumbing lives here; every computation is a library call.  The collectives run on the
 wire and statistics buffers in place (zero-copy views of the context's workspace), which are
 this GPU's own memory.
@@ -43,16 +46,21 @@ class DistributedRound:
         if local_grads.shape[0] != self.count:
             raise ValueError(f"rank {self.rank} owns {self.count} workers, got {local_grads.shape[0]} rows")
         ctx = self.ctx
-        ctx.fuse_local(local_grads)
-        if self.world > 1:
-            dist.all_reduce(ctx.local_stats(), op=dist.ReduceOp.SUM, group=self.group)
-        ctx.fuse_finish()
+        scalar_ref = ctx.norm == tng.NORM_MEAN          # every worker's own scalar: no fusion, no statistics
+        if not scalar_ref:
+            ctx.fuse_local(local_grads)
+            if self.world > 1:
+                dist.all_reduce(ctx.local_stats(), op=dist.ReduceOp.SUM, group=self.group)
+            ctx.fuse_finish()
         ctx.encode_local(local_grads, self.first, self.round)
         if self.world > 1:
             codes, scales = ctx.wire_views()
             lo, hi = self.first, self.first + self.count
             dist.all_gather_into_tensor(codes, codes[lo:hi].clone(), group=self.group)
             dist.all_gather_into_tensor(scales, scales[lo:hi].clone(), group=self.group)
+            if scalar_ref:                               # the scalars travel with the codes
+                means = ctx.wire_means_view()
+                dist.all_gather_into_tensor(means, means[lo:hi].clone(), group=self.group)
         ctx.decode_commit(out)
         self.round += 1
         return out

@@ -11,7 +11,7 @@ _PKG = Path(__file__).resolve().parent
 LIB_PATH = _PKG / "libtng.so"
 
 CODEC_SIGN1, CODEC_TERN2, CODEC_QSGD4 = 1, 2, 4
-NORM_NONE, NORM_DIFF, NORM_QUOT, NORM_COMB = 0, 1, 2, 3
+NORM_NONE, NORM_DIFF, NORM_QUOT, NORM_COMB, NORM_MEAN = 0, 1, 2, 3, 4
 SCALE_ABSMAX, SCALE_L2 = 0, 1
 FUSE_AUTO, FUSE_LAST, FUSE_MEAN, FUSE_LSQ, FUSE_HINDSIGHT = 0, 1, 2, 3, 4
 (OPT_BLOCK, OPT_QSGD_LEVELS, OPT_SCALE_KIND, OPT_SEED_LO, OPT_SEED_HI, OPT_FUSE_MODE, OPT_RIDGE, OPT_QUOT_EPS,
@@ -24,7 +24,7 @@ TILE = 128
 EXPORTS = [
     "tng_create", "tng_destroy", "tng_set_option", "tng_workspace_bytes", "tng_bind_workspace",
     "tng_push_reference", "tng_step", "tng_step_host", "tng_fuse", "tng_encode", "tng_decode_aggregate",
-    "tng_wire", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
+    "tng_wire", "tng_wire_means", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
     "tng_logistic_scratch_floats", "tng_logistic_grad", "tng_logistic_loss", "tng_rosenbrock_grad",
     "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static", "tng_state_bytes", "tng_save_state", "tng_load_state",
     "tng_fuse_local", "tng_local_stats", "tng_fuse_finish", "tng_encode_local", "tng_decode_commit",
@@ -74,6 +74,7 @@ def lib():
         L.tng_encode.argtypes = [vp, vp, u64, vp, u32, vp]
         L.tng_decode_aggregate.argtypes = [vp, vp, vp, vp]
         L.tng_wire.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t), C.POINTER(vp), C.POINTER(C.c_size_t)]
+        L.tng_wire_means.argtypes = [vp, C.POINTER(vp)]
         L.tng_reference.argtypes = [vp, C.POINTER(vp)]
         L.tng_history.argtypes = [vp, u32, C.POINTER(vp)]
         L.tng_stats.argtypes = [vp, C.POINTER(Stats)]
@@ -262,6 +263,15 @@ class Context:
         wpw, spw = C.c_size_t(), C.c_size_t()
         _check(lib().tng_wire(self._h, C.byref(cp), C.byref(wpw), C.byref(sp), C.byref(spw)), "tng_wire")
         return cp.value, wpw.value, sp.value, spw.value
+
+    def wire_means_view(self):
+        """Zero-copy view of the M scalar references (NORM_MEAN), for collectives."""
+        p = C.c_void_p()
+        _check(lib().tng_wire_means(self._h, C.byref(p)), "tng_wire_means")
+        return _view(p.value, (self.M,), torch.float32)
+
+    def wire_means(self):
+        return self.wire_means_view().clone()
 
     def reference(self):
         p = C.c_void_p()
