@@ -77,10 +77,15 @@ typedef enum {
     TNG_OPT_QUOT_EPS = 7,    /* floor of |r| relative to its tile maximum, quotient form.  Default 2^-4. */
     TNG_OPT_TIMING = 8,      /* 1 = record CUDA events around every stage of tng_step.  Default 0. */
     TNG_OPT_HOST_STAGING = 9,/* 1 = reserve device staging so tng_step_host can be used.  Default 0. */
-    TNG_OPT_REF_EVERY = 10   /* refresh cadence of the reference (Sec. 3.1, last paragraph; Sec. 4.1 refreshes
+    TNG_OPT_REF_EVERY = 10,  /* refresh cadence of the reference (Sec. 3.1, last paragraph; Sec. 4.1 refreshes
                                 every 16 iterations): tng_step fuses a new reference in rounds t with
                                 t % value == 0 and reuses the previous one in between; the ring still
                                 receives every aggregate.  1..65536, default 1. */
+    TNG_OPT_COORD_OFFSET = 11 /* the context holds coordinates [offset, offset + d) of a longer vector (one
+                                slice per GPU): only the Philox counters see the offset, so that the slices
+                                code exactly what one context over the whole vector would.  A multiple of 128
+                                and of the scale block; not with one scale per vector nor TNG_NORM_MEAN, which
+                                need the whole vector.  Default 0. */
 } tng_option;
 
 #define TNG_MAX_WORKERS 64
@@ -200,6 +205,16 @@ tng_status tng_decode_aggregate(tng_ctx* ctx, const float* ref_dev, float* out_d
 tng_status tng_fuse_local(tng_ctx* ctx, const float* grads_dev, uint64_t ld, uint32_t m_count, void* stream);
 /* Borrowed device pointer to the block to all-reduce (rhs[16], grad_sq) and its length. */
 tng_status tng_local_stats(tng_ctx* ctx, double** sums_dev, size_t* count);
+/* The other way to spread one round over GPUs: every process holds ALL M workers but only the
+ * coordinates [offset, offset + d) of every vector (TNG_OPT_COORD_OFFSET), ring and wire included.
+ * Encoding and decoding are local to a slice; the only coupling is the fusion statistics, which
+ * are sums over coordinates:
+ *   tng_fuse_local      Gram, rhs sums and grad_sq over the local coordinates
+ *   [all-reduce (sum) of the tng_local_stats_all block: 273 doubles on the device]
+ *   tng_fuse_finish     divide by M, solve, combine -> the slice of the reference
+ *   tng_encode_local    (m_first = 0, m_count = M), tng_decode_commit: no exchange of the wire
+ * Borrowed device pointer to G (16 x 16, row-major), c (16), grad_sq (1), contiguous. */
+tng_status tng_local_stats_all(tng_ctx* ctx, double** sums_dev, size_t* count);
 tng_status tng_fuse_finish(tng_ctx* ctx, void* stream);
 /* step: the Philox step counter; pass the round number (tng_stats' rounds). */
 tng_status tng_encode_local(tng_ctx* ctx, const float* grads_dev, uint64_t ld, uint32_t m_first, uint32_t m_count,

@@ -28,6 +28,7 @@ struct tng_ctx {
     uint64_t block_opt = 128;
     int levels = 7, scale_kind = 0, fuse_mode = TNG_FUSE_AUTO, timing = 0, host_staging = 0;
     uint32_t ref_every = 1;
+    uint64_t coord_offset = 0;
     uint32_t seed_lo = 0, seed_hi = 0;
     double ridge = 1e-6;
     float quot_eps = 0.0625f;
@@ -111,6 +112,7 @@ void size_ctx(tng_ctx* c) {
     g.wpw = g.ntile * 4u * (uint64_t)c->codec;
     g.M = c->M; g.codec = c->codec; g.norm = c->norm; g.scale_kind = c->scale_kind; g.levels = c->levels;
     g.seed_lo = c->seed_lo; g.seed_hi = c->seed_hi; g.quot_eps = c->quot_eps;
+    g.tile0 = c->coord_offset / TNG_TILE;
     size_t off = 0;
     c->off_ring = off;      off += align_up((size_t)c->K * c->d_pad * sizeof(float));
     c->off_ref = off;       off += align_up((size_t)c->d_pad * sizeof(float));
@@ -132,6 +134,10 @@ void size_ctx(tng_ctx* c) {
 tng_status ensure_ready(tng_ctx* c, cudaStream_t st) {
     c->last_stream = st;
     if (c->ws_ready) return TNG_OK;
+    if (c->coord_offset != 0) {   // a slice of a longer vector: nothing may need the whole of it
+        if (c->block_opt == 0 || c->norm == TNG_NORM_MEAN) return TNG_ERR_UNSUPPORTED;
+        if (c->coord_offset % c->block_opt != 0) return TNG_ERR_INVALID_ARG;
+    }
     size_ctx(c);
     TNG_CUDA(c, cudaGetDevice(&c->device));
     int sms = 0;
@@ -371,6 +377,9 @@ tng_status tng_set_option(tng_ctx* c, tng_option key, double value) {
         case TNG_OPT_HOST_STAGING:
             if (value != 0 && value != 1) return TNG_ERR_INVALID_ARG;
             c->host_staging = (int)value; return TNG_OK;
+        case TNG_OPT_COORD_OFFSET:
+            if (value < 0 || value > 281474976710656.0 || value != floor(value) || fmod(value, (double)TNG_TILE) != 0.0) return TNG_ERR_INVALID_ARG;
+            c->coord_offset = (uint64_t)value; return TNG_OK;
         case TNG_OPT_REF_EVERY:
             if (value < 1 || value > 65536 || value != floor(value)) return TNG_ERR_INVALID_ARG;
             c->ref_every = (uint32_t)value; return TNG_OK;
@@ -532,8 +541,9 @@ tng_status tng_fuse_local(tng_ctx* c, const float* grads_dev, uint64_t ld, uint3
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
-    // the block the caller adds up over the ranks: rhs[16] and grad_sq; zero when this mode has none
-    TNG_CUDA(c, cudaMemsetAsync(c->fb()->gram + kGramRhs, 0, (kMaxK + 1) * sizeof(double), st));
+    // the block the caller adds up over the ranks (rhs[16] and grad_sq, or all of it when the ranks hold
+    // slices of the coordinates): zero wherever this round's statistics pass writes nothing
+    TNG_CUDA(c, cudaMemsetAsync(c->fb()->gram, 0, kGramDoubles * sizeof(double), st));
     const int mode = c->effective_mode();
     if (c->k == 0 || (mode != TNG_FUSE_LSQ && mode != TNG_FUSE_HINDSIGHT)) return TNG_OK;
     const float* rows[kMaxK];
@@ -550,6 +560,14 @@ tng_status tng_local_stats(tng_ctx* c, double** sums_dev, size_t* count) {
     if (!c->ws_ready) return TNG_ERR_STATE;
     *sums_dev = c->fb()->gram + kGramRhs;
     *count = (size_t)kMaxK + 1;
+    return TNG_OK;
+}
+
+tng_status tng_local_stats_all(tng_ctx* c, double** sums_dev, size_t* count) {
+    if (!c || !sums_dev || !count) return TNG_ERR_INVALID_ARG;
+    if (!c->ws_ready) return TNG_ERR_STATE;
+    *sums_dev = c->fb()->gram;
+    *count = (size_t)kGramDoubles;
     return TNG_OK;
 }
 

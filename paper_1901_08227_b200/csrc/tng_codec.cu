@@ -33,6 +33,7 @@ struct EncodeArgs {
     uint32_t* pipe_error;
     uint64_t d, ntile, block;
     uint64_t tile_begin;   // first tile this launch handles (the staged kernel takes the ones before it)
+    uint64_t tile0;        // tile index of local tile 0 within the whole vector: only the Philox counters see it
     uint32_t ld, nblk, wpw;
     uint32_t M, step;
     uint32_t m_base;   // worker index of row 0 (Philox counter word); the wire pointers are already offset
@@ -261,7 +262,7 @@ __device__ __forceinline__ void encode_tile(const EncodeArgs& a, const float* s_
         op = make_norm_op<NORM>(r, r2, a.quot_eps);
     }
     const uint64_t blk = (PHASE == kPhaseQuant) ? (T * kTile) / a.block : T;
-    const uint64_t q = T * 32u + (uint32_t)lane;                 // Philox counter of the lane's four coordinates
+    const uint64_t q = (T + a.tile0) * 32u + (uint32_t)lane;     // Philox counter of the lane's four coordinates
     const uint32_t q_lo = (uint32_t)q, q_hi = (uint32_t)(q >> 32);
     uint32_t rmax = 0;                                           // largest scale bit pattern of the tile
     // batches of rows; the next batch is in flight while the current one is encoded
@@ -364,7 +365,7 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
     uint32_t it = 0;
     for (uint64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
         const uint64_t T = c * kEncPipeWarps + (uint32_t)warp;
-        const uint64_t q = T * 32u + (uint32_t)lane;
+        const uint64_t q = (T + a.tile0) * 32u + (uint32_t)lane;
         const uint32_t q_lo = (uint32_t)q, q_hi = (uint32_t)(q >> 32);
         // ---- the reference(s) of the tile
         float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
@@ -961,7 +962,7 @@ cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grad
         for (int j = 0; j < fusion->k; ++j) a.hist[j] = fusion->rows[j];
     }
     a.grads = grads; a.ref = ref; a.codes = codes; a.scales = scales; a.tile_stat = tile_stat;
-    a.nonfinite = &fb->nonfinite; a.pipe_error = &fb->pipe_error; a.tile_begin = 0;
+    a.nonfinite = &fb->nonfinite; a.pipe_error = &fb->pipe_error; a.tile_begin = 0; a.tile0 = g.tile0;
     a.ld = (uint32_t)ld; a.d = g.d; a.ntile = g.ntile; a.nblk = (uint32_t)g.nblk; a.block = g.block; a.wpw = (uint32_t)g.wpw;
     a.M = g.M; a.step = step; a.m_base = m_base; a.levels = g.levels; a.pow24 = 1u << 24;
     a.quot_eps = g.quot_eps;

@@ -39,6 +39,7 @@ struct CodecGeom {
     int codec, norm, scale_kind, levels;
     uint32_t seed_lo, seed_hi;
     float quot_eps;
+    uint64_t tile0;      // index of the first tile within the whole vector (a context that holds a slice of it)
 };
 
 // ---- fusion (tng_fuse.cu) ---------------------------------------------------

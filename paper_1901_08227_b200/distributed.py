@@ -64,3 +64,48 @@ class DistributedRound:
         ctx.decode_commit(out)
         self.round += 1
         return out
+
+
+def coord_range(rank: int, world: int, d: int, block: int = 128):
+    """Coordinates [first, first + count) of `rank` when every rank holds a slice of all vectors:
+    slices are whole scale blocks (multiples of 128 coordinates), the last one takes the ragged end."""
+    if block < 128 or block % 128 != 0:
+        raise ValueError("slices need a scale block that is a multiple of 128 coordinates")
+    units = -(-d // block)
+    per = -(-units // world)
+    first = min(rank * per * block, d)
+    count = min(first + per * block, d) - first
+    if count <= 0:
+        raise ValueError(f"d = {d} is too short for {world} ranks of whole {block}-coordinate blocks")
+    return first, count
+
+
+class CoordShardedRound:
+    """The other split: every rank holds all M workers but only its slice of the coordinates (ring
+    and wire included).  `ctx` is a context of the slice's length created with
+    ``coord_offset=first`` (so that it draws the random numbers of its coordinates of the whole
+    vector).  Coding and decoding are local; the fusion statistics are sums over coordinates:
+
+        fuse_local -> all-reduce of 273 doubles (Gram, rhs, grad_sq) -> fuse_finish
+                   -> encode_local (all M workers) -> decode_commit
+
+    Every rank ends up with its slice of what one context over the whole vector computes."""
+
+    def __init__(self, ctx: tng.Context, group=None):
+        self.ctx, self.group = ctx, group
+        self.world = dist.get_world_size(group) if group is not None else 1
+        self.round = 0
+
+    def step(self, grads_slice: torch.Tensor, out: torch.Tensor | None = None):
+        """grads_slice: (M, count) — this rank's coordinates of every worker's gradient."""
+        ctx = self.ctx
+        if grads_slice.shape[0] != ctx.M:
+            raise ValueError(f"expected the rows of all {ctx.M} workers, got {grads_slice.shape[0]}")
+        ctx.fuse_local(grads_slice)
+        if self.world > 1:
+            dist.all_reduce(ctx.local_stats_all(), op=dist.ReduceOp.SUM, group=self.group)
+        ctx.fuse_finish()
+        ctx.encode_local(grads_slice, 0, self.round)
+        ctx.decode_commit(out)
+        self.round += 1
+        return out

@@ -15,7 +15,7 @@ NORM_NONE, NORM_DIFF, NORM_QUOT, NORM_COMB, NORM_MEAN = 0, 1, 2, 3, 4
 SCALE_ABSMAX, SCALE_L2 = 0, 1
 FUSE_AUTO, FUSE_LAST, FUSE_MEAN, FUSE_LSQ, FUSE_HINDSIGHT = 0, 1, 2, 3, 4
 (OPT_BLOCK, OPT_QSGD_LEVELS, OPT_SCALE_KIND, OPT_SEED_LO, OPT_SEED_HI, OPT_FUSE_MODE, OPT_RIDGE, OPT_QUOT_EPS,
- OPT_TIMING, OPT_HOST_STAGING, OPT_REF_EVERY) = range(11)
+ OPT_TIMING, OPT_HOST_STAGING, OPT_REF_EVERY, OPT_COORD_OFFSET) = range(12)
 (OK, ERR_INVALID_ARG, ERR_STATE, ERR_ALLOC, ERR_CUDA, ERR_NONFINITE, ERR_UNSUPPORTED) = range(7)
 MAX_HISTORY = 16
 TILE = 128
@@ -27,7 +27,7 @@ EXPORTS = [
     "tng_wire", "tng_wire_means", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
     "tng_logistic_scratch_floats", "tng_logistic_grad", "tng_logistic_loss", "tng_rosenbrock_grad",
     "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static", "tng_state_bytes", "tng_save_state", "tng_load_state",
-    "tng_fuse_local", "tng_local_stats", "tng_fuse_finish", "tng_encode_local", "tng_decode_commit",
+    "tng_fuse_local", "tng_local_stats", "tng_local_stats_all", "tng_fuse_finish", "tng_encode_local", "tng_decode_commit",
 ]
 
 
@@ -93,6 +93,7 @@ def lib():
         L.tng_load_state.argtypes = [vp, vp, C.c_size_t, vp]
         L.tng_fuse_local.argtypes = [vp, vp, u64, u32, vp]
         L.tng_local_stats.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
+        L.tng_local_stats_all.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
         L.tng_fuse_finish.argtypes = [vp, vp]
         L.tng_encode_local.argtypes = [vp, vp, u64, u32, u32, u32, vp]
         L.tng_decode_commit.argtypes = [vp, vp, vp]
@@ -136,7 +137,8 @@ class Context:
 
     _OPTS = {"block": OPT_BLOCK, "qsgd_levels": OPT_QSGD_LEVELS, "scale_kind": OPT_SCALE_KIND,
              "seed_lo": OPT_SEED_LO, "seed_hi": OPT_SEED_HI, "fuse_mode": OPT_FUSE_MODE, "ridge": OPT_RIDGE,
-             "quot_eps": OPT_QUOT_EPS, "timing": OPT_TIMING, "host_staging": OPT_HOST_STAGING, "ref_every": OPT_REF_EVERY}
+             "quot_eps": OPT_QUOT_EPS, "timing": OPT_TIMING, "host_staging": OPT_HOST_STAGING, "ref_every": OPT_REF_EVERY,
+             "coord_offset": OPT_COORD_OFFSET}
 
     def __init__(self, d, M, K, codec, norm, workspace=None, **options):
         self.d, self.M, self.K, self.codec, self.norm = int(d), int(M), int(K), int(codec), int(norm)
@@ -219,6 +221,12 @@ class Context:
         """Zero-copy float64 view of the block to all-reduce (sum) between fuse_local and fuse_finish."""
         p, n = C.c_void_p(), C.c_size_t()
         _check(lib().tng_local_stats(self._h, C.byref(p), C.byref(n)), "tng_local_stats")
+        return _view(p.value, (n.value,), torch.float64)
+
+    def local_stats_all(self) -> torch.Tensor:
+        """The same for ranks that hold slices of the coordinates: Gram, rhs and grad_sq (273 doubles)."""
+        p, n = C.c_void_p(), C.c_size_t()
+        _check(lib().tng_local_stats_all(self._h, C.byref(p), C.byref(n)), "tng_local_stats_all")
         return _view(p.value, (n.value,), torch.float64)
 
     def fuse_finish(self):

@@ -138,3 +138,79 @@ def test_one_rank_over_nccl():
     finally:
         if created:
             dist.destroy_process_group()
+
+
+# ---------------------------------------------------------------------------------------------
+# the other split: every rank holds all workers but a slice of the coordinates
+def sliced_round(ctxs, bounds, grads, t, outs):
+    for c, (lo, n) in zip(ctxs, bounds):
+        c.fuse_local(grads[:, lo:lo + n])
+    total = sum(c.local_stats_all().clone() for c in ctxs)      # the all-reduce of Gram, rhs, grad_sq
+    for c in ctxs:
+        c.local_stats_all().copy_(total)
+        c.fuse_finish()
+    for c, (lo, n), o in zip(ctxs, bounds, outs):
+        c.encode_local(grads[:, lo:lo + n], 0, t)
+        c.decode_commit(o)
+
+
+@pytest.mark.parametrize("mode,K", [(tng.FUSE_LAST, 1), (tng.FUSE_MEAN, 3), (tng.FUSE_LSQ, 4), (tng.FUSE_HINDSIGHT, 3)])
+@pytest.mark.parametrize("norm,codec,B,d", [(tng.NORM_QUOT, tng.CODEC_TERN2, 128, 2048 * 40 + 128 * 3 + 8),
+                                            (tng.NORM_DIFF, tng.CODEC_QSGD4, 256, 256 * 37 + 100),
+                                            (tng.NORM_COMB, tng.CODEC_SIGN1, 128, 128 * 50 + 4)])
+@pytest.mark.parametrize("P", [2, 3])
+def test_coordinate_slices_reproduce_the_round_over_the_whole_vector(mode, K, norm, codec, B, d, P):
+    M, steps = 4, 2 * K + 2
+    opts = dict(block=B, fuse_mode=mode, seed_lo=6, qsgd_levels=4)
+    bounds = [distributed.coord_range(p, P, d, B) for p in range(P)]
+    assert bounds[0][0] == 0 and sum(n for _, n in bounds) == d
+    ranks = [make_ctx(n, M, K, codec, norm, coord_offset=lo, **opts) for lo, n in bounds]
+    single = make_ctx(d, M, K, codec, norm, **opts)
+    orc = make_oracle(d, M, K, codec, norm, **opts)
+    outs = [torch.empty(n, device="cuda") for _, n in bounds]
+    out1 = torch.empty(d, device="cuda")
+    exact = mode in (tng.FUSE_LAST, tng.FUSE_MEAN)               # no statistics involved
+    for t, g in enumerate(drifting_grads(3, steps, M, d, "cuda", ld=d + (4 - d % 4) % 4)):
+        sliced_round(ranks, bounds, g, t, outs)
+        single.step(g, out1)
+        want = orc.step(to_np(g))
+        whole = torch.cat(outs)
+        ref = torch.cat([c.reference() for c in ranks])
+        if exact:
+            assert torch.equal(whole, out1), f"aggregate differs at round {t}"
+            assert same_values(to_np(whole), want)
+            codes1, scales1 = single.wire()
+            tpb = B // 128
+            for c, (lo, n) in zip(ranks, bounds):
+                codes, scales = c.wire()
+                w0, w1 = lo // 128 * 4 * codec, -(-(lo + n) // 128) * 4 * codec
+                assert torch.equal(codes, codes1[:, w0:w1]), f"codes differ at round {t}"
+                assert torch.equal(scales, scales1[:, lo // B:-(-(lo + n) // B)])
+        else:
+            assert rel_l2(to_np(ref), to_np(single.reference())) < 1e-5 or t == 0
+            a_s, a_1 = np.array(ranks[0].stats().alpha[:K]), np.array(single.stats().alpha[:K])
+            assert np.allclose(a_s, a_1, rtol=0, atol=1e-6 * max(1.0, np.abs(a_1).max()))
+            for c in ranks[1:]:                                   # every rank solved the same system
+                assert np.array_equal(np.array(c.stats().alpha[:K]), a_s)
+    for c in ranks:
+        st = c.stats()
+        assert st.rounds == steps and st.k == min(steps, K) and st.pipeline_error == 0
+
+
+def test_a_slice_needs_whole_blocks_and_no_whole_vector_quantities():
+    g = torch.randn(2, 1024, device="cuda")
+    with pytest.raises(tng.TngError) as e:
+        make_ctx(1024, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, coord_offset=100)         # not a multiple of 128
+    assert e.value.status == tng.ERR_INVALID_ARG
+    c = make_ctx(1024, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, block=256, coord_offset=128)  # not a multiple of the block
+    with pytest.raises(tng.TngError) as e:
+        c.step(g)
+    assert e.value.status == tng.ERR_INVALID_ARG
+    for kw, norm in ((dict(block=0), tng.NORM_DIFF), (dict(block=128), tng.NORM_MEAN)):
+        c = make_ctx(1024, 2, 2, tng.CODEC_TERN2, norm, coord_offset=1024, **kw)
+        with pytest.raises(tng.TngError) as e:
+            c.step(g)
+        assert e.value.status == tng.ERR_UNSUPPORTED
+    assert distributed.coord_range(1, 2, 1000, 128) == (512, 488)
+    with pytest.raises(ValueError):
+        distributed.coord_range(3, 4, 300, 128)

@@ -99,3 +99,130 @@ def test_the_wire_exchange_assembles_every_worker_slot_on_every_rank(tmp_path):
     import pytest
     with pytest.raises(ValueError):
         distributed.worker_range(0, 4, 6)
+
+
+# ---------------------------------------------------------------------------------------------
+# The round with the coordinates split over two gloo ranks.  The rank-local stages are played by
+# the oracle on the rank's slice (a stand-in with the context's method names), so that what is
+# under test is the driver: which block is all-reduced, in which order the stages run, and that
+# the slices put together are the round over the whole vector.
+class _OracleSliceContext:
+    def __init__(self, first, count, M, K, codec, norm, mode, seed):
+        import oracle
+        self.o, self.first, self.d, self.M, self.K = oracle, first, count, M, K
+        self.codec, self.norm, self.mode, self.seed = codec, norm, mode, seed
+        self.hist = []                                     # newest first
+        self.block = torch.zeros(273, dtype=torch.float64)
+        self.ref = np.zeros(count, dtype=np.float32)
+        self.alpha = np.zeros(K, dtype=np.float32)
+
+    def fuse_local(self, g):
+        self.block.zero_()
+        k = len(self.hist)
+        if k == 0 or self.mode != self.o.FUSE_LSQ:
+            return
+        G, c, gg = self.o.fuse_stats(self.hist, g.numpy())   # c and gg are means over the M rows
+        blk = self.block.numpy()
+        for i in range(k):
+            blk[i * 16:i * 16 + k] = G[i]
+        blk[256:256 + k] = c * self.M                      # the library hands out raw sums
+        blk[272] = gg * self.M
+
+    def local_stats_all(self):
+        return self.block
+
+    def fuse_finish(self):
+        k = len(self.hist)
+        if k == 0:
+            self.ref = np.zeros(self.d, dtype=np.float32)
+            return
+        if self.mode == self.o.FUSE_LSQ:
+            blk = self.block.numpy()
+            G = np.array([blk[i * 16:i * 16 + k] for i in range(k)])
+            _, a32, _ = self.o.fuse_solve(G, blk[256:256 + k] / self.M, 1e-6)
+        else:                                              # window average
+            a32 = np.full(k, np.float32(1.0) / np.float32(k), dtype=np.float32)
+        self.alpha = a32
+        self.ref = self.o.combine(self.hist, a32)
+
+    def encode_local(self, g, m_first, step):
+        assert m_first == 0
+        self.wire = self.o.encode(g.numpy(), self.ref, self.norm, self.codec, B=128, seed=(self.seed, 0), t=step,
+                                  coord_offset=self.first)
+
+    def decode_commit(self, out):
+        codes, scales = self.wire
+        res = self.o.decode_aggregate(codes, scales, self.d, self.ref, self.norm, self.codec, B=128)
+        self.hist = ([res] + self.hist)[:self.K]
+        if out is not None:
+            out.copy_(torch.from_numpy(res))
+
+
+def _sliced_main(rank, world, port, out_dir, mode):
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    import oracle
+    from paper_1901_08227_b200 import distributed
+    d, M, K, steps = 128 * 21 + 50, 3, 3, 6
+    first, count = distributed.coord_range(rank, world, d, 128)
+    ctx = _OracleSliceContext(first, count, M, K, oracle.CODEC_TERN2, oracle.NORM_DIFF, mode, seed=4)
+    drv = distributed.CoordShardedRound(ctx, group=dist.group.WORLD)
+    rng = np.random.default_rng(0)                         # the same gradients on both ranks
+    outs, alphas = [], []
+    mean = rng.standard_normal(d).astype(np.float32)
+    for t in range(steps):
+        mean = (0.9 * mean + 0.3 * rng.standard_normal(d)).astype(np.float32)
+        g = (mean[None] + 0.5 * rng.standard_normal((M, d))).astype(np.float32)
+        out = torch.empty(count)
+        drv.step(torch.from_numpy(np.ascontiguousarray(g[:, first:first + count])), out)
+        outs.append(out.numpy().copy())
+        alphas.append(ctx.alpha.copy())
+    np.save(Path(out_dir, f"sliced{rank}.npy"), np.stack(outs))
+    np.save(Path(out_dir, f"alpha{rank}.npy"), np.stack([np.resize(a, K) for a in alphas]))
+    dist.destroy_process_group()
+
+
+def _whole_vector_rounds(mode):
+    import oracle
+    d, M, K, steps = 128 * 21 + 50, 3, 3, 6
+    st = oracle.State(d, M, K, oracle.CODEC_TERN2, oracle.NORM_DIFF, fuse_mode=mode, seed_lo=4)
+    rng = np.random.default_rng(0)
+    outs = []
+    mean = rng.standard_normal(d).astype(np.float32)
+    for t in range(steps):
+        mean = (0.9 * mean + 0.3 * rng.standard_normal(d)).astype(np.float32)
+        g = (mean[None] + 0.5 * rng.standard_normal((M, d))).astype(np.float32)
+        outs.append(st.step(g))
+    return np.stack(outs)
+
+
+def test_coordinate_slices_over_two_gloo_ranks_make_the_whole_round(tmp_path):
+    import oracle
+    world = 2
+    for mode in (oracle.FUSE_MEAN, oracle.FUSE_LSQ):
+        mp.spawn(_sliced_main, args=(world, _free_port(), str(tmp_path), mode), nprocs=world, join=True)
+        got = np.concatenate([np.load(tmp_path / f"sliced{r}.npy") for r in range(world)], axis=1)
+        want = _whole_vector_rounds(mode)
+        a0, a1 = np.load(tmp_path / "alpha0.npy"), np.load(tmp_path / "alpha1.npy")
+        assert np.array_equal(a0, a1)                      # both ranks solved the summed statistics
+        if mode == oracle.FUSE_MEAN:
+            assert np.array_equal(got, want)               # no statistics: bit for bit
+        else:
+            # the Gram is summed slice by slice, so alpha may differ in the last bits: close, not equal
+            rel = np.linalg.norm(got.astype(np.float64) - want) / np.linalg.norm(want)
+            assert rel < 0.05 and np.array_equal(got[0], want[0])       # round 0: empty ring, exact
+            assert np.abs(a0).max() > 0.1                  # the statistics did arrive (alpha is not zero)
+
+
+def test_coordinate_ranges_are_whole_blocks_that_cover_the_vector():
+    from paper_1901_08227_b200 import distributed
+    import pytest
+    for d, world, block in ((1000, 2, 128), (128 * 9, 3, 256), (1 << 20, 8, 128), (129, 2, 128)):
+        spans = [distributed.coord_range(r, world, d, block) for r in range(world)]
+        assert spans[0][0] == 0 and spans[-1][0] + spans[-1][1] == d
+        for (lo, n), (lo2, _) in zip(spans, spans[1:]):
+            assert lo + n == lo2 and lo2 % block == 0
+    with pytest.raises(ValueError):
+        distributed.coord_range(0, 2, 1000, 100)
+    with pytest.raises(ValueError):
+        distributed.coord_range(1, 2, 128, 128)
