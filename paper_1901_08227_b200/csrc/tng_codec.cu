@@ -609,9 +609,8 @@ __device__ __forceinline__ void decode_worker(const uint32_t (&w)[4 * CODEC], co
 }
 
 // average over the M workers (Algorithm 1), put the reference back (Eq. 2 / Eq. 3), store
-template <int NORM, bool FULL>
-__device__ __forceinline__ void decode_finish(const DecodeArgs& a, const float (&acc)[4], const float4 r, const float4 r2,
-                                              const uint64_t i0) {
+template <int NORM>
+__device__ __forceinline__ float4 decode_denormalise(const DecodeArgs& a, const float (&acc)[4], const float4 r, const float4 r2) {
     float4 o;
     if (a.inv_m > 0.0f) {
         o.x = __fmul_rn(acc[0], a.inv_m); o.y = __fmul_rn(acc[1], a.inv_m); o.z = __fmul_rn(acc[2], a.inv_m); o.w = __fmul_rn(acc[3], a.inv_m);
@@ -629,13 +628,7 @@ __device__ __forceinline__ void decode_finish(const DecodeArgs& a, const float (
         o.x = __fadd_rn(__fmul_rn(den.x, o.x), r.x); o.y = __fadd_rn(__fmul_rn(den.y, o.y), r.y);
         o.z = __fadd_rn(__fmul_rn(den.z, o.z), r.z); o.w = __fadd_rn(__fmul_rn(den.w, o.w), r.w);
     }
-    if (FULL) {
-        if (a.out_a) *reinterpret_cast<float4*>(a.out_a + i0) = o;
-        if (a.out_b) *reinterpret_cast<float4*>(a.out_b + i0) = o;
-    } else {
-        if (a.out_a) store4(a.out_a, i0, a.d, o);
-        if (a.out_b) store4(a.out_b, i0, a.d, o);
-    }
+    return o;
 }
 
 // ---------------------------------------------------------------------------
@@ -726,20 +719,30 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
     constexpr uint32_t kRound = 32 / CODEC;
     const int lane = threadIdx.x & 31;
     DecodeSlot* slot = &slots[threadIdx.x >> 5];
-    const uint64_t nwarps = (uint64_t)gridDim.x * kDecWarps;
-    const uint64_t gwarp = (uint64_t)blockIdx.x * kDecWarps + (threadIdx.x >> 5);
-    const uint64_t nfull = a.d / kTile;
+    // Tile indices fit 32 bits (d <= 2^31), and so does every per-tile offset below: each address is
+    // then ONE 32 x 32 -> 64 multiply-add on a pointer that is either a kernel argument or a per-lane
+    // row pointer formed once (the lane's worker is the same for every tile).
+    const uint32_t nwarps = gridDim.x * kDecWarps;
+    const uint32_t gwarp = blockIdx.x * kDecWarps + (threadIdx.x >> 5);
+    const uint32_t nfull = (uint32_t)(a.d / kTile);
+    const uint32_t block32 = (uint32_t)a.block;
     const uint32_t pw = a.one << (31 - lane);
     const bool tiled = a.block == (uint64_t)kTile;
     const bool has_ref = (NORM != TNG_NORM_NONE) && (NORM != TNG_NORM_MEAN) && a.ref != nullptr;
+    const bool has_ref2 = (NORM == TNG_NORM_COMB) && a.ref2 != nullptr;
+    const bool to_a = a.out_a != nullptr, to_b = a.out_b != nullptr;
     const uint32_t n0 = a.M < kRound ? a.M : kRound;                 // workers of the first round
+    // first round: lane = worker * b + piece; the lane's own rows of the wire
+    const uint32_t my_m = (uint32_t)lane / CODEC, my_piece = (uint32_t)lane % CODEC;
+    const bool has_code = my_m < a.M, has_scale = (uint32_t)lane < n0;
+    const uint4* code_row = reinterpret_cast<const uint4*>(a.codes + (uint64_t)(has_code ? my_m : 0u) * a.wpw) + my_piece;
+    const float* scale_row = a.scales + (uint64_t)(has_scale ? (uint32_t)lane : 0u) * a.nblk;
+    const float4* ref4 = reinterpret_cast<const float4*>(a.ref) + lane;
+    const float4* ref24 = reinterpret_cast<const float4*>(a.ref2) + lane;
     // the sum starts from -0 so that (-0) + x == x bit for bit; the ternary path starts from +0
     // because it skips zero symbols and +0 is what the sum of skipped terms is
     const float z = (CODEC == TNG_CODEC_TERN2) ? 0.0f : -0.0f;
 
-    uint64_t T = a.tile_begin + gwarp;
-    uint4 cw = make_uint4(0u, 0u, 0u, 0u);
-    float sc = 0.0f;
     float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
     if (NORM == TNG_NORM_MEAN) {
         // what every element gets back: (1/M) sum_m mean(g^m), summed m ascending like the codes
@@ -749,29 +752,34 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
         r = make_float4(mbar, mbar, mbar, mbar);
     }
     const float4 r_const = r;
-    const bool has_ref2 = (NORM == TNG_NORM_COMB) && a.ref2 != nullptr;
-    if (T < nfull) {
-        decode_fetch<CODEC>(a, T, tiled ? T : (T * kTile) / a.block, 0, lane, cw, sc);
-        if (has_ref) r = *reinterpret_cast<const float4*>(a.ref + (T * kTile + (uint64_t)lane * 4u));
-        if (has_ref2) r2 = *reinterpret_cast<const float4*>(a.ref2 + (T * kTile + (uint64_t)lane * 4u));
-    }
+    // the three loads of tile t (first round of workers)
+    auto fetch = [&](const uint32_t t, uint4& cw, float& sc, float4& rr, float4& rr2) {
+        const uint32_t blk = tiled ? t : (t * (uint32_t)kTile) / block32;
+        cw = make_uint4(0u, 0u, 0u, 0u);
+        sc = 0.0f;
+        if (has_code) cw = __ldcs(code_row + (size_t)t * CODEC);
+        if (has_scale) sc = __ldcs(scale_row + blk);
+        if (has_ref) rr = ref4[(size_t)t * 32u];
+        if (has_ref2) rr2 = ref24[(size_t)t * 32u];
+    };
+
+    uint32_t T = (uint32_t)a.tile_begin + gwarp;
+    uint4 cw = make_uint4(0u, 0u, 0u, 0u);
+    float sc = 0.0f;
+    if (T < nfull) fetch(T, cw, sc, r, r2);
     for (; T < nfull; T += nwarps) {
         slot->cw[lane] = cw;
         slot->sc[lane] = sc;
         const float4 rcur = r, r2cur = r2;
         __syncwarp();
-        const uint64_t Tn = T + nwarps;
-        if (Tn < nfull) {                                            // next tile's loads go out now
-            decode_fetch<CODEC>(a, Tn, tiled ? Tn : (Tn * kTile) / a.block, 0, lane, cw, sc);
-            if (has_ref) r = *reinterpret_cast<const float4*>(a.ref + (Tn * kTile + (uint64_t)lane * 4u));
-            if (has_ref2) r2 = *reinterpret_cast<const float4*>(a.ref2 + (Tn * kTile + (uint64_t)lane * 4u));
-        }
+        const uint32_t Tn = T + nwarps;
+        if (Tn < nfull) fetch(Tn, cw, sc, r, r2);                     // next tile's loads go out now
         float acc[4] = {z, z, z, z};
         decode_round_any<CODEC>(slot, n0, a.levels, pw, lane, acc);
         for (uint32_t m0 = kRound; m0 < a.M; m0 += kRound) {         // more workers than one round holds
             uint4 cw2;
             float sc2;
-            decode_fetch<CODEC>(a, T, tiled ? T : (T * kTile) / a.block, m0, lane, cw2, sc2);
+            decode_fetch<CODEC>(a, T, tiled ? T : ((uint64_t)T * kTile) / a.block, m0, lane, cw2, sc2);
             __syncwarp();
             slot->cw[lane] = cw2;
             slot->sc[lane] = sc2;
@@ -779,10 +787,13 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
             decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
         }
         __syncwarp();                                                // slot is free again
-        decode_finish<NORM, true>(a, acc, rcur, r2cur, T * kTile + (uint64_t)lane * 4u);
+        const float4 o = decode_denormalise<NORM>(a, acc, rcur, r2cur);
+        const size_t at = (size_t)T * 32u + (uint32_t)lane;          // float4 index of the lane's coordinates
+        if (to_a) reinterpret_cast<float4*>(a.out_a)[at] = o;
+        if (to_b) reinterpret_cast<float4*>(a.out_b)[at] = o;
     }
     // the ragged last tile
-    if (nfull < a.ntile && gwarp == nfull % nwarps) {
+    if ((uint64_t)nfull < a.ntile && gwarp == nfull % nwarps) {
         const uint64_t Tr = nfull, i0 = Tr * kTile + (uint64_t)lane * 4u;
         const uint64_t blk = tiled ? Tr : (Tr * kTile) / a.block;
         float4 rr = (NORM == TNG_NORM_MEAN) ? r_const : make_float4(0.f, 0.f, 0.f, 0.f), rr2 = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -799,7 +810,9 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
             __syncwarp();
             decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
         }
-        decode_finish<NORM, false>(a, acc, rr, rr2, i0);
+        const float4 o = decode_denormalise<NORM>(a, acc, rr, rr2);
+        if (to_a) store4(a.out_a, i0, a.d, o);
+        if (to_b) store4(a.out_b, i0, a.d, o);
     }
 }
 
