@@ -74,7 +74,7 @@ def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True, ref_in_e
 # dram__bytes_read.sum + dram__bytes_write.sum per coordinate of the dominant kernel, from the ncu
 # capture summarised under profiles/ (taken at d = 2^24 and scaled by d: every kernel streams each
 # coordinate once).  None = the kernel changed after the capture.
-NCU_TRAFFIC_BYTES_PER_COORD = {"encode": 69.92, "dots": 64.35, "decode": 11.16}
+NCU_TRAFFIC_BYTES_PER_COORD = {"encode": 69.94, "dots": 64.25, "decode": 11.32}
 
 
 def measured_hbm_peak():
