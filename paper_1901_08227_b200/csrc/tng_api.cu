@@ -455,17 +455,18 @@ struct StateHeader {
     uint32_t k;
     uint64_t rounds;
     uint32_t has_ref, pad;
+    uint64_t coord_offset;
 };
 constexpr uint32_t kStateMagic = 0x53474e54u;   // "TNGS"
 
 void fill_header(const tng_ctx* c, StateHeader* h) {
     memset(h, 0, sizeof *h);
-    h->magic = kStateMagic; h->version = 1;
+    h->magic = kStateMagic; h->version = 2;
     h->d = c->d; h->M = c->M; h->K = c->K; h->codec = (uint32_t)c->codec; h->norm = (uint32_t)c->norm;
     h->block = c->block_opt; h->levels = (uint32_t)c->levels; h->scale_kind = (uint32_t)c->scale_kind;
     h->fuse_mode = (uint32_t)c->fuse_mode; h->seed_lo = c->seed_lo; h->seed_hi = c->seed_hi; h->ref_every = c->ref_every;
     h->ridge = c->ridge; h->quot_eps = c->quot_eps;
-    h->k = c->k; h->rounds = c->rounds; h->has_ref = 0;
+    h->k = c->k; h->rounds = c->rounds; h->has_ref = 0; h->coord_offset = c->coord_offset;
 }
 }  // namespace
 
@@ -504,7 +505,7 @@ tng_status tng_load_state(tng_ctx* c, const void* host_buf, size_t bytes, void* 
     StateHeader h, mine;
     memcpy(&h, host_buf, sizeof h);
     fill_header(c, &mine);
-    if (h.magic != kStateMagic || h.version != 1 || h.d != mine.d || h.M != mine.M || h.K != mine.K || h.codec != mine.codec ||
+    if (h.magic != kStateMagic || h.version != 2 || h.coord_offset != mine.coord_offset || h.d != mine.d || h.M != mine.M || h.K != mine.K || h.codec != mine.codec ||
         h.norm != mine.norm || h.block != mine.block || h.levels != mine.levels || h.scale_kind != mine.scale_kind ||
         h.fuse_mode != mine.fuse_mode || h.seed_lo != mine.seed_lo || h.seed_hi != mine.seed_hi || h.ref_every != mine.ref_every ||
         h.ridge != mine.ridge || h.quot_eps != mine.quot_eps || h.k > h.K || h.has_ref > 2 ||

@@ -63,6 +63,7 @@ def test_a_state_of_another_configuration_is_rejected():
     a.step(g)
     blob = a.save_state()
     for other in (make_ctx(1000, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=2),
+                  make_ctx(1000, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=1, coord_offset=1024),
                   make_ctx(1000, 2, 3, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=1),
                   make_ctx(1004, 2, 2, tng.CODEC_TERN2, tng.NORM_DIFF, seed_lo=1)):
         with pytest.raises(tng.TngError) as e:
@@ -74,3 +75,23 @@ def test_a_state_of_another_configuration_is_rejected():
     small = torch.empty(64, dtype=torch.uint8)
     st = tng.lib().tng_save_state(a._h, small.data_ptr(), small.numel(), None, 0)
     assert st == tng.ERR_ALLOC
+
+
+def test_a_state_with_the_scalar_reference_continues_bit_for_bit():
+    d, M, K = 2048 * 9 + 77, 3, 2
+    opts = dict(block=128, seed_lo=3)
+    a = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_MEAN, **opts)
+    grads = list(drifting_grads(4, 6, M, d, "cuda"))
+    for g in grads:
+        g += 0.5                                           # in place: the rows keep their padded stride
+    out = torch.empty(d, device="cuda")
+    for g in grads[:3]:
+        a.step(g, out)
+    blob = a.save_state()
+    b = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_MEAN, **opts)
+    b.load_state(blob)
+    out_b = torch.empty(d, device="cuda")
+    for g in grads[3:]:
+        a.step(g, out)
+        b.step(g, out_b)
+        assert torch.equal(out, out_b) and torch.equal(a.wire()[0], b.wire()[0]) and torch.equal(a.wire_means(), b.wire_means())
