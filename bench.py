@@ -208,7 +208,9 @@ def run_reference(args, name, cfg):
     print(json.dumps(line), flush=True)
 
 
-def time_cpu_baseline(cfg, enums, limit_s=12.0):
+def time_cpu_baseline(cfg, enums, limit_s=12.0, single_thread=True):
+    import numpy as np
+
     import oracle
     from paper_1901_08227_b200 import workloads
     norm, codec, fuse = enums
@@ -229,8 +231,26 @@ def time_cpu_baseline(cfg, enums, limit_s=12.0):
         if dt > limit_s or n >= 50:
             break
     per = dt / n
-    return {"value": M * d_s * 4 / per / 1e9, "unit": UNIT, "cores": oracle.omp_threads(), "kind": "oracle",
-            "sample": f"first {d_s} of {cfg['d']} coordinates per step, {n} steps, {per * 1e3:.1f} ms each"}
+    cores = oracle.omp_threads()
+    res = {"value": M * d_s * 4 / per / 1e9, "unit": UNIT, "cores": cores, "kind": "oracle",
+           "sample": f"first {d_s} of {cfg['d']} coordinates per step, {n} steps, {per * 1e3:.1f} ms each"}
+    if single_thread and cores > 1:
+        # the same oracle on one thread, on a shorter sample (a quarter of the coordinates, one step)
+        d_1 = max(d_s // 4, 1 << 14)
+        orc1 = oracle.State(d_1, M, K, codec, norm, block=cfg["block"], fuse_mode=fuse)
+        for j in range(K):
+            orc1.push_reference(np.ascontiguousarray(orc.history(K - 1 - j)[:d_1]))
+        g1 = np.ascontiguousarray(g[:, :d_1])
+        oracle.set_threads(1)
+        try:
+            t1 = time.perf_counter()
+            orc1.step(g1)
+            dt1 = time.perf_counter() - t1
+        finally:
+            oracle.set_threads(cores)
+        res["single_thread"] = {"value": M * d_1 * 4 / dt1 / 1e9, "unit": UNIT,
+                                "sample": f"first {d_1} coordinates, 1 step, {dt1 * 1e3:.0f} ms"}
+    return res
 
 
 # --------------------------------------------------------------------------------------

@@ -113,19 +113,20 @@ def lib():
         L.tngo_rosenbrock_value.argtypes = [_f32p, C.c_uint64]
         L.tngo_rosenbrock_grad.argtypes = [_f32p, C.c_uint64, _f32p, C.c_int, C.c_uint64, _f32p]
         L.tngo_sgd_update.argtypes = [_f32p, _f32p, C.c_uint64, C.c_float]
+        L.tngo_max_threads.restype = C.c_int
+        L.tngo_set_threads.argtypes = [C.c_int]
         _lib = L
     return _lib
 
 
 def omp_threads() -> int:
     """Threads the OpenMP loops of the oracle will use."""
-    env = os.environ.get("OMP_NUM_THREADS")
-    if env:
-        return int(env.split(",")[0])
-    try:
-        return len(os.sched_getaffinity(0))
-    except AttributeError:
-        return os.cpu_count() or 1
+    return int(lib().tngo_max_threads())
+
+
+def set_threads(n: int) -> None:
+    """Threads for the oracle's parallel loops from now on (timing only: no result depends on it)."""
+    lib().tngo_set_threads(int(n))
 
 
 # --------------------------------------------------------------------------- helpers

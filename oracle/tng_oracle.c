@@ -733,6 +733,18 @@ void tngo_rosenbrock_grad(const float* x, uint64_t d, const float* noise, int M,
     }
 }
 
+/* ------------------------------------------------------------------------- */
+/* how many threads the parallel loops use (timing only; results do not depend on it) */
+/* ------------------------------------------------------------------------- */
+#ifdef _OPENMP
+#include <omp.h>
+int tngo_max_threads(void) { return omp_get_max_threads(); }
+void tngo_set_threads(int n) { if (n > 0) omp_set_num_threads(n); }
+#else
+int tngo_max_threads(void) { return 1; }
+void tngo_set_threads(int n) { (void)n; }
+#endif
+
 void tngo_sgd_update(float* w, const float* v, uint64_t d, float eta) {
     for (uint64_t i = 0; i < d; ++i) {
         float stepv = eta * v[i];

@@ -158,6 +158,10 @@ void tngo_rosenbrock_grad(const float* x, uint64_t d, const float* noise, int M,
 /* w <- w - eta * v, one fp32 multiply and one fp32 subtraction per element. */
 void tngo_sgd_update(float* w, const float* v, uint64_t d, float eta);
 
+/* ---- threads of the parallel loops (for timing the oracle; no result depends on them) */
+int tngo_max_threads(void);
+void tngo_set_threads(int n);
+
 #ifdef __cplusplus
 }
 #endif
