@@ -162,6 +162,17 @@ __device__ __forceinline__ void encode_quantise(const EncodeArgs& a, const float
     }
 }
 
+// The operands worker m normalises with: the tile's, except for the scalar reference, where every
+// worker subtracts its own mean (Section 3.1).  Full tiles only (no element past the end).
+template <int NORM>
+__device__ __forceinline__ NormOp worker_op(const EncodeArgs& a, const NormOp& op, const uint32_t m) {
+    if (NORM != TNG_NORM_MEAN) return op;
+    NormOp o = op;
+    const float mu = __ldg(a.means + m);
+    o.a = make_float4(mu, mu, mu, mu);
+    return o;
+}
+
 template <int CODEC, int NORM, int SCALE, int PHASE, bool FULL>
 __device__ __forceinline__ bool encode_symbols(const EncodeArgs& a, const float4 g, const NormOp& op,
                                                const uint32_t m, const uint64_t T, const uint4 x, const uint64_t blk,
@@ -430,7 +441,8 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                         const int k = k0 + kk;
                         uint32_t w[kWords];
                         float R;
-                        encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g[k], op, m0 + k, T, x[kk], T, lane, 0xFu, w, R);
+                        encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g[k], worker_op<NORM>(a, op, m0 + k), m0 + k, T, x[kk], T, lane,
+                                                                               0xFu, w, R);
                         store_words_if<CODEC>(lane == k, my_codes, w);
                         my_R = (lane == k) ? R : my_R;
                     }
@@ -441,7 +453,7 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
                     uint32_t w[kWords];
                     float R;
                     const uint4 x = philox4x32_10_rk(q_lo, q_hi, a.m_base + m0 + k, a.step, a.rk);
-                    encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, op, m0 + k, T, x, T, lane, 0xFu, w, R);
+                    encode_symbols<CODEC, NORM, SCALE, kPhaseFused, true>(a, g, worker_op<NORM>(a, op, m0 + k), m0 + k, T, x, T, lane, 0xFu, w, R);
                     store_words_if<CODEC>((uint32_t)lane == k, my_codes, w);
                     my_R = ((uint32_t)lane == k) ? R : my_R;
                 }
@@ -862,7 +874,7 @@ cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t
         pa.rows.nrows = 0;
         if (FUSEREF) {
             for (int j = 0; j < a.hist_k; ++j) pa.rows.row[pa.rows.nrows++] = a.hist[j];
-        } else if (NORM != TNG_NORM_NONE && a.ref) {
+        } else if (NORM != TNG_NORM_NONE && NORM != TNG_NORM_MEAN && a.ref) {
             pa.rows.row[pa.rows.nrows++] = a.ref;
             if (NORM == TNG_NORM_COMB && a.ref2) pa.rows.row[pa.rows.nrows++] = a.ref2;
         }
@@ -882,9 +894,9 @@ cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t
 
 template <int CODEC, int NORM, int SCALE, int PHASE>
 cudaError_t encode_launch(const EncodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
-    if constexpr (PHASE == kPhaseFused && NORM != TNG_NORM_MEAN) {   // the scalar reference takes the direct kernels
-        if (NORM != TNG_NORM_NONE && a.hist_k > 0)
-            return encode_launch_tiles<CODEC, NORM, SCALE, (NORM != TNG_NORM_NONE)>(a, sm_count, st, launches);
+    if constexpr (PHASE == kPhaseFused) {
+        if (NORM != TNG_NORM_NONE && NORM != TNG_NORM_MEAN && a.hist_k > 0)
+            return encode_launch_tiles<CODEC, NORM, SCALE, (NORM != TNG_NORM_NONE && NORM != TNG_NORM_MEAN)>(a, sm_count, st, launches);
         return encode_launch_tiles<CODEC, NORM, SCALE, false>(a, sm_count, st, launches);
     } else {
         ++*launches;
