@@ -74,6 +74,10 @@ def algorithmic_bytes_per_coord(M, K, bits, block, fuse, user_out=True, ref_in_e
 # dram__bytes_read.sum + dram__bytes_write.sum per coordinate of the dominant kernel, from the ncu
 # capture summarised under profiles/ (taken at d = 2^24 and scaled by d: every kernel streams each
 # coordinate once).  None = the kernel changed after the capture.
+# integer/logic-pipe instructions the staged encode kernel issues per tile and worker (ternary, quotient
+# form; from the opcode histogram of the same capture: 22 logic ops, 9 float compares, 8 ballots, 6 integer
+# compares, 4 conversions, 3 integer adds, 3 max, 2 selects, 3 others)
+ALU_PIPE_INSTR_PER_TILE_WORKER = 60
 NCU_TRAFFIC_BYTES_PER_COORD = {"encode": 69.94, "dots": 64.25, "decode": 11.32}
 
 
@@ -341,6 +345,16 @@ def run_ours(args, name, cfg):
     roofline = {"bound": "hbm", "kernel": dominant, "achieved": kernels[dominant]["GBps"], "peak": peak, "unit": "GB/s",
                 "frac": kernels[dominant]["frac_of_measured"], "peak_source": peak_src, "traffic": traffic,
                 "algorithmic_bytes_per_launch": per_coord[dominant] * d}
+    if profiled and dominant == "encode" and clocks.get("sm_mhz"):
+        # The encode pass is the one kernel that is closer to an arithmetic roof than to HBM: its busiest unit
+        # is the integer/logic pipe, which takes one warp instruction every two cycles per SM partition
+        # (4 partitions x 148 SMs).  The opcode histogram of the ncu capture gives about 60 such
+        # instructions per tile (128 coordinates) and worker; stated beside the HBM figure, not instead of it.
+        alu_peak = 0.5 * 4 * 148 * clocks["sm_mhz"] * 1e6
+        alu_rate = ALU_PIPE_INSTR_PER_TILE_WORKER * (d / 128.0) * M / (kernels["encode"]["ms"] * 1e-3)
+        roofline["alu_pipe"] = {"bound": "alu", "achieved": alu_rate / 1e9, "peak": alu_peak / 1e9, "unit": "G warp-instr/s",
+                                "frac": alu_rate / alu_peak,
+                                "peak_source": "0.5 warp-instr/cycle x 4 partitions x 148 SMs x sampled SM clock"}
     step_bytes = sum(per_coord.values()) * d
     step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
 
