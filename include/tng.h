@@ -235,6 +235,15 @@ tng_status tng_reference(tng_ctx* ctx, const float** ref_dev);
 /* h_{j+1}: j = 0 is the newest stored aggregate; j < k. */
 tng_status tng_history(tng_ctx* ctx, uint32_t j, const float** vec_dev);
 
+/* ---- self-test of the bounded waits ------------------------------------------------ */
+/* The staged kernels wait on shared-memory barriers with a poll limit; when a wait runs out the
+ * kernel records it, returns, and tng_stats reports TNG_ERR_CUDA with pipeline_error set.  This
+ * call exercises exactly that path without disturbing the context: a one-block kernel waits
+ * (same wait routine, limit of 1024 polls) on a barrier that nothing ever completes and writes
+ * what happened to a scratch word of the workspace.  *gave_up_host = 1 when the wait ended by
+ * its limit, as it must.  Synchronises the stream.  The context stays usable. */
+tng_status tng_selftest_bounded_wait(tng_ctx* ctx, uint32_t* gave_up_host, void* stream);
+
 /* ---- fusion statistics without any allocation ------------------------------- */
 /* (No counterpart in the paper: this is a packaging of the statistics pass of tng_fuse.)
  * For callers that cannot allocate device memory -- a process whose device memory is

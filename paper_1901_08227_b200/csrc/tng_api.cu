@@ -7,6 +7,7 @@
 #include <new>
 
 #include "tng_internal.h"
+#include "tng_pipeline.cuh"
 
 using namespace tng;
 
@@ -315,6 +316,19 @@ tng_status step_impl(tng_ctx* c, const float* grads, uint64_t ld, float* out, cu
     return TNG_OK;
 }
 
+// nothing ever arrives on this barrier: the wait has to end by its poll limit
+__global__ void bounded_wait_selftest_kernel(uint32_t* outcome) {
+    __shared__ uint64_t bar;
+    const uint32_t b = tng::smem_u32(&bar);
+    if (threadIdx.x == 0) {
+        tng::mbar_init(b, 1);
+        tng::mbar_init_fence();
+    }
+    __syncthreads();
+    const bool completed = tng::mbar_wait_limited(b, 0u, 1024);
+    if (threadIdx.x == 0) *outcome = completed ? 2u : 1u;
+}
+
 }  // namespace
 
 // =========================================================================================
@@ -561,6 +575,23 @@ tng_status tng_local_stats(tng_ctx* c, double** sums_dev, size_t* count) {
     if (!c->ws_ready) return TNG_ERR_STATE;
     *sums_dev = c->fb()->gram + kGramRhs;
     *count = (size_t)kMaxK + 1;
+    return TNG_OK;
+}
+
+tng_status tng_selftest_bounded_wait(tng_ctx* c, uint32_t* gave_up_host, void* stream) {
+    if (!c || !gave_up_host) return TNG_ERR_INVALID_ARG;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    uint32_t* word = reinterpret_cast<uint32_t*>(c->partials());   // scratch between launches of the statistics pass
+    TNG_CUDA(c, cudaMemsetAsync(word, 0, sizeof(uint32_t), st));
+    bounded_wait_selftest_kernel<<<1, 32, 0, st>>>(word);
+    TNG_CUDA(c, cudaGetLastError());
+    uint32_t outcome = 0;
+    TNG_CUDA(c, cudaMemcpyAsync(&outcome, word, sizeof outcome, cudaMemcpyDeviceToHost, st));
+    TNG_CUDA(c, cudaStreamSynchronize(st));
+    *gave_up_host = (outcome == 1u) ? 1u : 0u;
+    c->launches += 1;
     return TNG_OK;
 }
 

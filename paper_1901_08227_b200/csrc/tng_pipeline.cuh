@@ -66,11 +66,12 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
     return ok != 0;
 }
 // bounded wait; false = gave up
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) {
-    for (int i = 0; i < kSpinLimit; ++i)
+__device__ __forceinline__ bool mbar_wait_limited(uint32_t bar, uint32_t parity, int limit) {
+    for (int i = 0; i < limit; ++i)
         if (mbar_try_wait(bar, parity)) return true;
     return false;
 }
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity) { return mbar_wait_limited(bar, parity, kSpinLimit); }
 // Same for the producer thread, which has nothing else to do: each poll may sleep up to
 // `kProducerNapNs` inside the hardware wait, so that its polling does not take issue slots
 // from the compute warps of its scheduler.  Still bounded.

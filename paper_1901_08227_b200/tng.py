@@ -27,7 +27,7 @@ EXPORTS = [
     "tng_wire", "tng_wire_means", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
     "tng_logistic_scratch_floats", "tng_logistic_grad", "tng_logistic_loss", "tng_rosenbrock_grad",
     "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static", "tng_state_bytes", "tng_save_state", "tng_load_state",
-    "tng_fuse_local", "tng_local_stats", "tng_local_stats_all", "tng_fuse_finish", "tng_encode_local", "tng_decode_commit",
+    "tng_selftest_bounded_wait", "tng_fuse_local", "tng_local_stats", "tng_local_stats_all", "tng_fuse_finish", "tng_encode_local", "tng_decode_commit",
 ]
 
 
@@ -94,6 +94,7 @@ def lib():
         L.tng_fuse_local.argtypes = [vp, vp, u64, u32, vp]
         L.tng_local_stats.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
         L.tng_local_stats_all.argtypes = [vp, C.POINTER(vp), C.POINTER(C.c_size_t)]
+        L.tng_selftest_bounded_wait.argtypes = [vp, C.POINTER(C.c_uint32), vp]
         L.tng_fuse_finish.argtypes = [vp, vp]
         L.tng_encode_local.argtypes = [vp, vp, u64, u32, u32, u32, vp]
         L.tng_decode_commit.argtypes = [vp, vp, vp]
@@ -222,6 +223,12 @@ class Context:
         p, n = C.c_void_p(), C.c_size_t()
         _check(lib().tng_local_stats(self._h, C.byref(p), C.byref(n)), "tng_local_stats")
         return _view(p.value, (n.value,), torch.float64)
+
+    def selftest_bounded_wait(self) -> bool:
+        """True when a wait on a barrier that nothing completes ended by its poll limit (as it must)."""
+        out = C.c_uint32(0)
+        _check(lib().tng_selftest_bounded_wait(self._h, C.byref(out), _stream()), "tng_selftest_bounded_wait")
+        return out.value == 1
 
     def local_stats_all(self) -> torch.Tensor:
         """The same for ranks that hold slices of the coordinates: Gram, rhs and grad_sq (273 doubles)."""
