@@ -175,13 +175,15 @@ tng_status tng_fuse(tng_ctx* ctx, const float* grads_dev, uint64_t ld, void* str
  * "compute R, sample z, transmit"): normalise against ref_dev (d floats, device; NULL = the
  * context's reference), one scale per block, stochastic rounding, bit packing -> the wire
  * (tng_wire).  `step` is the Philox step counter (tng_step passes the round number).  With
- * TNG_NORM_COMB the second reference is always the context's own (from the last fusion). */
+ * TNG_NORM_COMB the second reference is always the context's own (from the last fusion).  With
+ * TNG_NORM_MEAN ref_dev is ignored: the workers' means are computed first (tng_wire_means). */
 tng_status tng_encode(tng_ctx* ctx, const float* grads_dev, uint64_t ld, const float* ref_dev,
                       uint32_t step, void* stream);
 /* Decode + aggregate (Algorithm 1 "the main server averages", with Eq. 2 / Eq. 3's v = ref + r /
  * ref . r): unpack the M code streams of the wire, v^m = R^m * symbol, a = (sum_m v^m) / M in
- * fp32 (m ascending), de-normalise against ref_dev (NULL = context's).  Writes out_dev (d floats,
- * device); does not touch the ring. */
+ * fp32 (m ascending), de-normalise against ref_dev (NULL = context's; ignored with TNG_NORM_MEAN,
+ * which adds the average of the wire's M scalars instead).  Writes out_dev (d floats, device);
+ * does not touch the ring. */
 tng_status tng_decode_aggregate(tng_ctx* ctx, const float* ref_dev, float* out_dev, void* stream);
 
 /* ---- the same round with the workers on different GPUs ------------------------------- */
