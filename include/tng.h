@@ -149,6 +149,16 @@ tng_status tng_step(tng_ctx* ctx, const float* grads_dev, uint64_t ld, float* ag
  * TNG_OPT_HOST_STAGING = 1.  Pinned host memory makes the copies asynchronous and fast. */
 tng_status tng_step_host(tng_ctx* ctx, const float* grads_host, uint64_t ld, float* agg_out_host,
                          void* stream);
+/* The same without waiting: the copy of the aggregate to agg_out_host runs on a stream of the
+ * library's own, so that in a sequence of calls it overlaps the next call's copy of the rows to the
+ * device (the link carries both directions at once).  grads_host may be reused once the call has
+ * returned and `stream` has passed its copy (tng_host_wait also guarantees that for every earlier
+ * call); agg_out_host holds the aggregate only after tng_host_wait.  Pinned host memory is needed
+ * for any overlap. */
+tng_status tng_step_host_async(tng_ctx* ctx, const float* grads_host, uint64_t ld, float* agg_out_host,
+                               void* stream);
+/* Blocks until every copy started by tng_step_host_async has finished. */
+tng_status tng_host_wait(tng_ctx* ctx);
 
 /* ---- state save / resume ----------------------------------------------------- */
 /* The state a context carries between rounds is the ring, the round counter and (with a refresh

@@ -58,6 +58,10 @@ struct tng_ctx {
     int last_cuda_error = 0;
     uint64_t launches = 0;
     unsigned long long nonfinite_reported = 0;
+    // tng_step_host_async: the library's own stream for the copies back to the host
+    cudaStream_t copy_stream = nullptr;
+    cudaEvent_t ev_round_done = nullptr, ev_copied = nullptr;
+    bool copy_pending = false;
     // timing
     cudaEvent_t ev[kTimedRounds][kStages + 1];
     bool ev_created = false;
@@ -351,6 +355,12 @@ tng_status tng_create(tng_ctx** out, uint64_t d, uint32_t M, uint32_t K, tng_cod
 void tng_destroy(tng_ctx* c) {
     if (!c) return;
     if (c->ws_ready) cudaStreamSynchronize(c->last_stream);
+    if (c->copy_stream) {
+        cudaStreamSynchronize(c->copy_stream);
+        cudaEventDestroy(c->ev_round_done);
+        cudaEventDestroy(c->ev_copied);
+        cudaStreamDestroy(c->copy_stream);
+    }
     if (c->ev_created)
         for (int r = 0; r < kTimedRounds; ++r)
             for (int s = 0; s <= kStages; ++s) cudaEventDestroy(c->ev[r][s]);
@@ -454,6 +464,41 @@ tng_status tng_step_host(tng_ctx* c, const float* grads_host, uint64_t ld, float
     if (s != TNG_OK) return s;
     TNG_CUDA(c, cudaMemcpyAsync(agg_out_host, c->stage_o(), c->d * sizeof(float), cudaMemcpyDeviceToHost, st));
     TNG_CUDA(c, cudaStreamSynchronize(st));
+    return TNG_OK;
+}
+
+tng_status tng_step_host_async(tng_ctx* c, const float* grads_host, uint64_t ld, float* agg_out_host, void* stream) {
+    if (!c || !grads_host || !agg_out_host || ld < c->d || ld > 0xFFFFFFFCull) return TNG_ERR_INVALID_ARG;
+    if (!c->host_staging) return TNG_ERR_STATE;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    if (!c->copy_stream) {
+        TNG_CUDA(c, cudaStreamCreateWithFlags(&c->copy_stream, cudaStreamNonBlocking));
+        TNG_CUDA(c, cudaEventCreateWithFlags(&c->ev_round_done, cudaEventDisableTiming));
+        TNG_CUDA(c, cudaEventCreateWithFlags(&c->ev_copied, cudaEventDisableTiming));
+    }
+    TNG_CUDA(c, cudaMemcpy2DAsync(c->stage_g(), c->d_pad * sizeof(float), grads_host, ld * sizeof(float),
+                                  c->d * sizeof(float), c->M, cudaMemcpyHostToDevice, st));
+    // the previous aggregate must have left the staging buffer before this round's decode rewrites it;
+    // the rows above do not wait for that, which is where the two directions overlap
+    if (c->copy_pending) TNG_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied, 0));
+    s = step_impl(c, c->stage_g(), c->d_pad, c->stage_o(), st);
+    if (s != TNG_OK) return s;
+    TNG_CUDA(c, cudaEventRecord(c->ev_round_done, st));
+    TNG_CUDA(c, cudaStreamWaitEvent(c->copy_stream, c->ev_round_done, 0));
+    TNG_CUDA(c, cudaMemcpyAsync(agg_out_host, c->stage_o(), c->d * sizeof(float), cudaMemcpyDeviceToHost, c->copy_stream));
+    TNG_CUDA(c, cudaEventRecord(c->ev_copied, c->copy_stream));
+    c->copy_pending = true;
+    return TNG_OK;
+}
+
+tng_status tng_host_wait(tng_ctx* c) {
+    if (!c) return TNG_ERR_INVALID_ARG;
+    if (!c->copy_pending) return TNG_OK;
+    TNG_CUDA(c, cudaStreamSynchronize(c->last_stream));   // the rows of the last call have been read
+    TNG_CUDA(c, cudaEventSynchronize(c->ev_copied));
+    c->copy_pending = false;
     return TNG_OK;
 }
 

@@ -23,7 +23,7 @@ TILE = 128
 # every symbol include/tng.h declares
 EXPORTS = [
     "tng_create", "tng_destroy", "tng_set_option", "tng_workspace_bytes", "tng_bind_workspace",
-    "tng_push_reference", "tng_step", "tng_step_host", "tng_fuse", "tng_encode", "tng_decode_aggregate",
+    "tng_push_reference", "tng_step", "tng_step_host", "tng_step_host_async", "tng_host_wait", "tng_fuse", "tng_encode", "tng_decode_aggregate",
     "tng_wire", "tng_wire_means", "tng_reference", "tng_history", "tng_stats", "tng_status_string", "tng_last_cuda_error",
     "tng_logistic_scratch_floats", "tng_logistic_grad", "tng_logistic_loss", "tng_rosenbrock_grad",
     "tng_rosenbrock_value", "tng_sgd_update", "tng_gram_static", "tng_state_bytes", "tng_save_state", "tng_load_state",
@@ -70,6 +70,8 @@ def lib():
         L.tng_push_reference.argtypes = [vp, vp, vp]
         L.tng_step.argtypes = [vp, vp, u64, vp, vp]
         L.tng_step_host.argtypes = [vp, vp, u64, vp, vp]
+        L.tng_step_host_async.argtypes = [vp, vp, u64, vp, vp]
+        L.tng_host_wait.argtypes = [vp]
         L.tng_fuse.argtypes = [vp, vp, u64, vp]
         L.tng_encode.argtypes = [vp, vp, u64, vp, u32, vp]
         L.tng_decode_aggregate.argtypes = [vp, vp, vp, vp]
@@ -195,6 +197,17 @@ class Context:
         _check(lib().tng_step_host(self._h, grads_host.data_ptr(), grads_host.stride(0), out_host.data_ptr(), _stream()),
                "tng_step_host")
         return out_host
+
+    def step_host_async(self, grads_host: torch.Tensor, out_host: torch.Tensor):
+        """step_host without waiting: out_host holds the aggregate after host_wait()."""
+        if grads_host.is_cuda or out_host.is_cuda or grads_host.dtype != torch.float32 or grads_host.stride(1) != 1:
+            raise TypeError("step_host_async takes host float32 tensors")
+        _check(lib().tng_step_host_async(self._h, grads_host.data_ptr(), grads_host.stride(0), out_host.data_ptr(), _stream()),
+               "tng_step_host_async")
+        return out_host
+
+    def host_wait(self):
+        _check(lib().tng_host_wait(self._h), "tng_host_wait")
 
     def state_bytes(self) -> int:
         n = C.c_size_t()

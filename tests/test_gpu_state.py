@@ -95,3 +95,28 @@ def test_a_state_with_the_scalar_reference_continues_bit_for_bit():
         a.step(g, out)
         b.step(g, out_b)
         assert torch.equal(out, out_b) and torch.equal(a.wire()[0], b.wire()[0]) and torch.equal(a.wire_means(), b.wire_means())
+
+
+def test_rounds_on_host_buffers_with_and_without_waiting_agree():
+    d, M, K, steps = 2048 * 9 + 333, 3, 2, 5
+    opts = dict(block=128, seed_lo=4, host_staging=1)
+    a = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, **opts)
+    b = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, **opts)
+    c = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, block=128, seed_lo=4)
+    grads = [g.cpu().contiguous().pin_memory() for g in drifting_grads(6, steps, M, d, "cuda", ld=d)]
+    outs_a = [torch.empty(d).pin_memory() for _ in range(steps)]
+    outs_b = [torch.empty(d).pin_memory() for _ in range(steps)]
+    for g, o in zip(grads, outs_a):
+        a.step_host(g, o)
+    for g, o in zip(grads, outs_b):
+        b.step_host_async(g, o)                            # nothing is waited for until the end
+    b.host_wait()
+    out = torch.empty(d, device="cuda")
+    for g, oa, ob in zip(grads, outs_a, outs_b):
+        ld = (d + 3) // 4 * 4
+        gd = torch.zeros((M, ld), device="cuda")
+        gd[:, :d] = g.cuda()
+        c.step(gd[:, :d], out)
+        assert torch.equal(oa, ob) and torch.equal(out.cpu(), oa)
+    b.host_wait()                                          # nothing pending: returns at once
+    assert a.stats().rounds == b.stats().rounds == steps
