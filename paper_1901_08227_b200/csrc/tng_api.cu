@@ -460,6 +460,7 @@ tng_status tng_step_host(tng_ctx* c, const float* grads_host, uint64_t ld, float
     if (s != TNG_OK) return s;
     TNG_CUDA(c, cudaMemcpy2DAsync(c->stage_g(), c->d_pad * sizeof(float), grads_host, ld * sizeof(float),
                                   c->d * sizeof(float), c->M, cudaMemcpyHostToDevice, st));
+    if (c->copy_pending) TNG_CUDA(c, cudaStreamWaitEvent(st, c->ev_copied, 0));   // an earlier tng_step_host_async still copying out
     s = step_impl(c, c->stage_g(), c->d_pad, c->stage_o(), st);
     if (s != TNG_OK) return s;
     TNG_CUDA(c, cudaMemcpyAsync(agg_out_host, c->stage_o(), c->d * sizeof(float), cudaMemcpyDeviceToHost, st));
