@@ -1,0 +1,57 @@
+"""GPU parity on randomly drawn configurations: vector lengths around tile, chunk and block
+boundaries, worker counts on both sides of a decode round (32 / b workers) and of a pipeline fill
+(8 rows), every codec, normalisation, scale kind and block size, with and without a refresh cadence.
+Whole rounds against the oracle, bit for bit, with the fusion modes whose reference involves no
+statistics (delayed gradient, window average); the draws are fixed by the seed."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import codes_np, drifting_grads, make_ctx, make_oracle, round_up4, same_bits, same_values, to_np
+from paper_1901_08227_b200 import tng
+
+
+def draw(seed):
+    rng = np.random.default_rng(1000 + seed)
+    kind = rng.integers(0, 4)
+    if kind == 0:
+        d = int(rng.integers(1, 700))
+    elif kind == 1:
+        d = int(128 * rng.integers(1, 60) + rng.choice([-1, 0, 1, 3, 64, 127]))
+    elif kind == 2:
+        d = int(2048 * rng.integers(8, 14) + rng.choice([-129, -1, 0, 1, 128, 130, 2047]))   # staged kernels + tails
+    else:
+        d = int(rng.integers(700, 40000))
+    d = max(d, 1)
+    M = int(rng.choice([1, 2, 3, 5, 7, 8, 9, 12, 16, 17, 33, 64], p=[.1, .1, .1, .1, .1, .15, .1, .05, .05, .05, .05, .05]))
+    K = int(rng.integers(1, 6))
+    codec = int(rng.choice([tng.CODEC_SIGN1, tng.CODEC_TERN2, tng.CODEC_QSGD4]))
+    norm = int(rng.choice([tng.NORM_NONE, tng.NORM_DIFF, tng.NORM_QUOT, tng.NORM_COMB, tng.NORM_MEAN]))
+    block = int(rng.choice([0, 128, 128, 128, 256, 384, 1024]))
+    mode = int(rng.choice([tng.FUSE_LAST, tng.FUSE_MEAN]))
+    opts = dict(block=block, fuse_mode=mode, seed_lo=int(rng.integers(0, 2 ** 31)), seed_hi=int(rng.integers(0, 2 ** 31)),
+                qsgd_levels=int(rng.integers(1, 8)), scale_kind=int(rng.integers(0, 2)), ref_every=int(rng.choice([1, 1, 2, 3])))
+    return d, M, K, codec, norm, opts
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(120))
+def test_random_configuration_rounds_are_bit_exact(seed):
+    d, M, K, codec, norm, opts = draw(seed)
+    ctx = make_ctx(d, M, K, codec, norm, **opts)
+    orc = make_oracle(d, M, K, codec, norm, **opts)
+    out = torch.empty(d, device="cuda")
+    what = f"d={d} M={M} K={K} codec={codec} norm={norm} {opts}"
+    for t, g in enumerate(drifting_grads(seed, K + 3, M, d, "cuda", ld=round_up4(d) + 4 * (seed % 3))):
+        if norm == tng.NORM_MEAN:
+            g += 0.25 * (1 + seed % 5)
+        ctx.step(g, out)
+        want = orc.step(to_np(g))
+        codes, scales = ctx.wire()
+        assert np.array_equal(codes_np(codes), orc.codes()), f"codes differ at round {t}: {what}"
+        assert same_values(to_np(scales), orc.scales()), f"scales differ at round {t}: {what}"
+        if norm == tng.NORM_MEAN:
+            assert same_bits(to_np(ctx.wire_means()), orc.means()), f"means differ at round {t}: {what}"
+        assert same_values(to_np(out), want), f"aggregate differs at round {t}: {what}"
+    st = ctx.stats()
+    assert st.pipeline_error == 0 and st.rounds == K + 3, what
