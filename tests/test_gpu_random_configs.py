@@ -55,3 +55,47 @@ def test_random_configuration_rounds_are_bit_exact(seed):
         assert same_values(to_np(out), want), f"aggregate differs at round {t}: {what}"
     st = ctx.stats()
     assert st.pipeline_error == 0 and st.rounds == K + 3, what
+
+
+def draw_fusion(seed):
+    rng = np.random.default_rng(5000 + seed)
+    k = int(rng.integers(1, 17))                                  # 9..16 take the cross-block statistics kernel
+    M = int(rng.choice([1, 2, 3, 5, 8, 9, 16, 24, 64]))
+    d = int(rng.choice([rng.integers(1, 3000), 1024 * rng.integers(16, 40) + rng.choice([-1, 0, 1, 515]), rng.integers(3000, 60000)]))
+    mode = int(rng.choice([tng.FUSE_LSQ, tng.FUSE_HINDSIGHT]))
+    return k, M, d, mode
+
+
+@pytest.mark.gpu
+@pytest.mark.parametrize("seed", range(40))
+def test_random_fusion_statistics_and_coefficients(seed):
+    """Gram, right-hand side, coefficients and fused reference of randomly drawn histories against
+    the oracle, within the tolerances of the fusion tests (1e-10 on the fp64 Gram, 1e-5 on alpha
+    and the reference)."""
+    import oracle
+    from gpu_util import rel_l2
+    from paper_1901_08227_b200 import workloads
+    k, M, d, mode = draw_fusion(seed)
+    ctx = make_ctx(d, M, k, tng.CODEC_TERN2, tng.NORM_DIFF, fuse_mode=mode)
+    orc = make_oracle(d, M, k, tng.CODEC_TERN2, tng.NORM_DIFF, fuse_mode=mode)
+    traj = workloads.AR1Trajectory(seed, d, device="cuda", rho=0.5)   # weakly correlated: a well-conditioned Gram
+    for _ in range(k):
+        h = traj.advance().contiguous()
+        ctx.push_reference(h)
+        orc.push_reference(to_np(h))
+    g = traj.worker_grads(M, 0.5, ld=round_up4(d) + 4)
+    ctx.fuse(g)
+    orc.fuse(to_np(g))
+    st = ctx.stats()
+    what = f"k={k} M={M} d={d} mode={mode}"
+    assert st.k == k and st.solver_fallback == orc.fallback, what
+    if orc.fallback:
+        return
+    G = np.array(st.gram[:]).reshape(16, 16)[:k, :k]
+    oG, oc, ogg = orc.gram()
+    assert rel_l2(G, oG) < 1e-10, what
+    if mode == tng.FUSE_LSQ:
+        assert rel_l2(np.array(st.rhs[:k]), oc) < 1e-6 and st.grad_sq == pytest.approx(ogg, rel=1e-6), what
+    alpha = np.array(st.alpha[:k])
+    assert np.allclose(alpha, orc.alpha().astype(np.float64)[:k], rtol=0, atol=1e-5 * max(1.0, np.abs(alpha).max())), what
+    assert rel_l2(to_np(ctx.reference()), orc.ref()) < 1e-5 or not orc.ref().any(), what
