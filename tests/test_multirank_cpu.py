@@ -70,6 +70,12 @@ def test_algorithmic_bytes_of_the_round():
     assert sum(per.values()) == 148.5
     split = bench.algorithmic_bytes_per_coord(8, 8, 2, 128, "lsq", ref_in_encode=False)
     assert split["combine"] == 36.0 and split["encode"] == 38.25
+    comb = bench.algorithmic_bytes_per_coord(8, 8, 2, 128, "lsq", norm="comb")     # a second reference written and read
+    assert comb["encode"] == 74.25 and comb["decode"] == 18.25
+    scalar = bench.algorithmic_bytes_per_coord(8, 8, 2, 128, "lsq", norm="mean")   # no fusion, the rows read twice
+    assert set(scalar) == {"encode", "decode"} and scalar["encode"] == 66.25 and scalar["decode"] == 10.25
+    last = bench.algorithmic_bytes_per_coord(8, 8, 2, 128, "last")                 # the reference is a ring slot: no combine
+    assert "dots" not in last and last["encode"] == 38.25
 
 
 def _gather_main(rank, world, port, out_dir):
