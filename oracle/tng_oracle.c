@@ -344,8 +344,10 @@ static uint32_t quant_sign1(float v, float R, float u) {
     return (u * R < thr) ? 1u : 0u;
 }
 /* s-level stochastic uniform quantiser (QSGD, Alistarh et al. 2017):
- * a = (|v|/R) s, level floor(a) or floor(a)+1 with probability frac(a).  Both
- * scale kinds give |v| <= R, so a <= s and the level never exceeds s.
+ * a = (|v|/R) s, level floor(a) or floor(a)+1 with probability frac(a), and never
+ * above s: the quantiser has the levels 0..s only.  The bound matters when the L2
+ * scale underestimates |v| (v*v subnormal, so sqrtf(fl(v*v)) < |v| and a > s);
+ * without it level s+1 would spill into the sign bit of the 4-bit symbol.
  * symbol bits 0..2 = level, bit 3 = negative. */
 static uint32_t quant_qsgd4(float v, float R, float u, int s) {
     float q = fabsf(v) / R;
@@ -353,6 +355,7 @@ static uint32_t quant_qsgd4(float v, float R, float u, int s) {
     float l = floorf(a);
     float f = a - l;
     int L = (int)l + ((u < f) ? 1 : 0);
+    if (L > s) L = s;
     uint32_t neg = (L > 0 && v < 0.0f) ? 1u : 0u;
     return (uint32_t)L | (neg << 3);
 }

@@ -197,6 +197,49 @@ def test_qsgd_l2_scale_unbiased():
     _check_moments(v, mean, var, (Rv / 7) ** 2 * f * (1 - f), S, Rv)
 
 
+def test_qsgd_level_never_exceeds_s_when_the_l2_scale_underestimates():
+    # The cited s-level quantiser has levels 0..s and nothing above.  With the L2 scale and a block whose
+    # squares are subnormal, sqrt(fl(v*v)) < |v|, so |v|/R > 1 and floor(a) + 1 would be s + 1: in the
+    # 4-bit symbol that spills into the sign bit.  The level is therefore bounded by s.
+    s = 7
+    for x in (1e-22, 3e-22, -1e-22, -3e-22):
+        v = np.zeros(128, dtype=np.float32)
+        v[37] = x
+        R = np.sqrt(np.float32(v[37] * v[37]))
+        assert R > 0 and abs(np.float32(x)) / R > 1.0          # the premise of the case
+        for t in range(200):
+            codes, sc = oracle.encode(v[None], None, NORM_NONE, CODEC_QSGD4, B=128, s=s, scale_kind=SCALE_L2, t=t)
+            assert sc[0, 0] == R
+            sym = unpack_symbols(codes[0], 128, 4)
+            assert (sym & 7)[37] <= s
+            assert (sym[37] >> 3) == (1 if x < 0 else 0)           # sign bit = (v < 0), not a spilt level bit
+            assert (sym & 7)[37] == s                               # a >= s: the top level, always
+            assert not np.delete(sym, 37).any()
+            out = oracle.decode_aggregate(codes, sc, 128, None, NORM_NONE, CODEC_QSGD4, B=128, s=s)
+            assert (out[37] > 0) == (x > 0) and abs(out[37]) == np.float32(np.float32(s) * np.float32(R / np.float32(s)))
+
+
+def test_qsgd_level_bound_changes_nothing_in_the_normal_range():
+    # in the normal range a <= s up to rounding; when a == s exactly, floor(a) = s and frac = 0, so the
+    # bound is never active: the symbols equal an independent numpy restatement without it
+    rng = np.random.default_rng(77)
+    d, s = 512, 7
+    v = rng.standard_normal(d).astype(np.float32)
+    for kind in (SCALE_ABSMAX, SCALE_L2):
+        for t in range(20):
+            codes, sc = oracle.encode(v[None], None, NORM_NONE, CODEC_QSGD4, B=128, s=s, scale_kind=kind, t=t, seed=(3, 9))
+            sym = unpack_symbols(codes[0], d, 4)
+            R = np.repeat(sc[0], 128)[:d]
+            a = (np.abs(v) / R).astype(np.float32) * np.float32(s)
+            l = np.floor(a)
+            f = (a - l).astype(np.float32)
+            u = np.array([oracle.coord_uniform(3, 9, i, 0, t) for i in range(d)], dtype=np.float32)
+            L = l.astype(np.int64) + (u < f)
+            assert L.max() <= s
+            assert np.array_equal(sym & 7, L.astype(np.uint32))
+            assert np.array_equal(sym >> 3, ((L > 0) & (v < 0)).astype(np.uint32))
+
+
 # ------------------------------------------------------------------ scales
 def test_absmax_scale_per_block_and_per_vector():
     rng = np.random.default_rng(3)
