@@ -102,7 +102,8 @@ typedef struct {
     uint64_t rounds;         /* completed rounds (the Philox step counter) */
     double bits_per_coord;   /* b + 32/B + 64 K/d */
     double alpha[TNG_MAX_HISTORY];                     /* coefficients of the last fusion */
-    double gram[TNG_MAX_HISTORY * TNG_MAX_HISTORY];    /* k x k, row-major (LSQ / HINDSIGHT) */
+    double gram[TNG_MAX_HISTORY * TNG_MAX_HISTORY];    /* G[a][b] at gram[a * TNG_MAX_HISTORY + b], a, b < k: the
+                                                          row stride is always 16, whatever k (LSQ / HINDSIGHT) */
     double rhs[TNG_MAX_HISTORY];                       /* <h_i, mean gradient> */
     double grad_sq;          /* (1/M) sum_m ||g^m||^2 of the last fusion */
     double cnz;              /* estimate of C_nz = sum_m||g^m - r||^2 / sum_m||g^m||^2; NaN if unknown */
@@ -128,12 +129,14 @@ tng_status tng_set_option(tng_ctx* ctx, tng_option key, double value);
 /* Device bytes the context needs (ring K*d, reference, codes, scales, reduction scratch). */
 tng_status tng_workspace_bytes(tng_ctx* ctx, size_t* bytes);
 /* Use caller-owned device memory (256-byte aligned, >= tng_workspace_bytes) instead of an
- * internal cudaMalloc.  Must come before the first device call.  Contents are cleared lazily
- * on `stream` of the first device call. */
+ * internal cudaMalloc.  Must come before the first device call.  Only the small state block
+ * (statistics, flags, counters) is cleared, on `stream` of the first device call; the ring, the
+ * wire and the scratch areas are left as found and are written before they are read. */
 tng_status tng_bind_workspace(tng_ctx* ctx, void* dev_ptr, size_t bytes);
 
 /* ---- the round ------------------------------------------------------------- */
-/* Seed the ring with a vector (Sec. 4.2: "initialise the reference with a full gradient"). */
+/* Seed the ring with a vector (the start-up of Sec. 4.2, where the first reference is a gradient
+ * computed in full rather than zeros). */
 tng_status tng_push_reference(tng_ctx* ctx, const float* vec_dev, void* stream);
 /* One round of Algorithm 1 on M gradient rows (row m at grads_dev + m*ld, device memory):
  * fusion of the reference from the ring (Sec. 3.1, criterion of Prop. 2), r(w_t) = Q[normalised
@@ -276,7 +279,10 @@ tng_status tng_selftest_bounded_wait(tng_ctx* ctx, uint32_t* gave_up_host, void*
  * The first call on each device looks up the array's device address (with that device
  * current); make that first call outside any stream capture.  All calls share the one
  * array: it is cleared where it must start at zero, but two calls that overlap on the
- * GPU (different streams, different threads) race and give wrong sums. */
+ * GPU (different streams, different threads) race and give wrong sums.
+ * The call never waits for the GPU, so a failure that only shows there is reported in the
+ * output: if a bounded wait of the staged statistics kernel gave up, all k*k+k+1 outputs
+ * are NaN (the sums would be incomplete). */
 #define TNG_STATIC_MAX_HISTORY 8
 #define TNG_STATIC_SCRATCH_BYTES (320 * 1024)
 tng_status tng_gram_static(const float* const* rows_dev, uint32_t k, uint64_t d, const float* grads_dev,

@@ -120,8 +120,9 @@ __device__ __forceinline__ float encode_tile_stat(const float (&v)[4]) {
 
 // Stochastic rounding of the lane's four values with scale R; x = the lane's Philox call,
 // word c for coordinate 4j+c.  The ballots leave every code word of the tile in every lane.
-// A scale that is zero, NaN or infinite needs no special case: u*0 < 0, NaN < x and inf < x
-// are all false, and (int)NaN is 0, so every symbol of such a block is the zero symbol.
+// A scale that is NaN or infinite needs no special case, nor does a zero max-scale (the block is
+// then all zeros): u*0 < 0, NaN < x and inf < x are all false, and (int)NaN is 0, so every symbol
+// of such a block is the zero symbol.  The caller replaces a zero L2 scale by NaN.
 //
 // The integer/logic pipe is the busy one in the encode kernels (Philox xors, compares,
 // ballots), so work that can run on the multiplier pipe is put there: addresses are
@@ -147,12 +148,13 @@ __device__ __forceinline__ void encode_quantise(const EncodeArgs& a, const float
             const bool plus = live && (__fmul_rn(u, R) < thr);
             w[c] = __ballot_sync(kFullMask, plus);
         } else {
-            // s-level: a = (|v|/R) s; level floor(a) (+1 with probability frac(a))
+            // s-level: a = (|v|/R) s; level floor(a) (+1 with probability frac(a)), never above s (an L2
+            // scale can fall short of |v| when the squares are subnormal; level s+1 would reach the sign plane)
             const float qv = __fdiv_rn(fabsf(v[c]), R);
             const float av = __fmul_rn(qv, (float)a.levels);
             const float lv = floorf(av);
             const float fv = __fsub_rn(av, lv);
-            const int L = live ? ((int)lv + ((u < fv) ? 1 : 0)) : 0;
+            const int L = live ? min((int)lv + ((u < fv) ? 1 : 0), a.levels) : 0;
             const bool neg = (L > 0) && (v[c] < 0.0f);
             w[c * 4 + 0] = __ballot_sync(kFullMask, L & 1);
             w[c * 4 + 1] = __ballot_sync(kFullMask, L & 2);
@@ -190,7 +192,10 @@ __device__ __forceinline__ bool encode_symbols(const EncodeArgs& a, const float4
     } else {
         R = __ldg(a.scales + (uint64_t)m * a.nblk + blk);
     }
-    encode_quantise<CODEC, FULL>(a, v, R, x, valid, w);
+    // An L2 scale can be zero although the block is not (all squares underflow): the comparisons below
+    // would then fire on u*0 < |v|.  A NaN in R's place makes every one of them false: the zero symbol.
+    const float Rq = (SCALE == 1 && !(R > 0.0f)) ? __int_as_float(0x7fc00000) : R;
+    encode_quantise<CODEC, FULL>(a, v, Rq, x, valid, w);
     return true;
 }
 
@@ -844,9 +849,14 @@ int persistent_grid(Kern kern, uint64_t ntile, int sm_count) {
 
 template <int CODEC, int NORM, int SCALE, int PHASE, bool FUSEREF>
 cudaError_t encode_launch_direct(const EncodeArgs& a, int sm_count, cudaStream_t st) {
-    static int per_tiles_grid = 0;   // grid when tiles are plentiful
+    static PerDevice<int> cached;   // grid when tiles are plentiful, per device
     auto kern = encode_kernel<CODEC, NORM, SCALE, PHASE, FUSEREF>;
-    if (per_tiles_grid == 0) per_tiles_grid = persistent_grid(kern, ~0ull >> 8, sm_count);
+    const int slot = device_slot();
+    int per_tiles_grid = slot >= 0 ? cached.v[slot] : 0;
+    if (per_tiles_grid == 0) {
+        per_tiles_grid = persistent_grid(kern, ~0ull >> 8, sm_count);
+        if (slot >= 0) cached.v[slot] = per_tiles_grid;
+    }
     const uint64_t want = (a.ntile - a.tile_begin + 7) / 8;
     const int grid = (int)(want < (uint64_t)per_tiles_grid ? (want ? want : 1) : (uint64_t)per_tiles_grid);
     kern<<<grid, kCodecThreads, 0, st>>>(a);
@@ -861,12 +871,13 @@ cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t
     EncodeArgs a = a0;
     a.tile_begin = 0;
     if (nchunks >= kEncPipeMinChunks) {
-        static bool configured = false;   // opt in to the large dynamic shared memory once per instantiation
+        static PerDevice<bool> configured;   // opt in to the large dynamic shared memory once per instantiation and device
         auto kern = encode_pipe_kernel<CODEC, NORM, SCALE, FUSEREF>;
-        if (!configured) {
+        const int slot = device_slot();
+        if (slot < 0 || !configured.v[slot]) {
             cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EncGeom::kSmemBytes);
             if (e != cudaSuccess) return e;
-            configured = true;
+            if (slot >= 0) configured.v[slot] = true;
         }
         EncodePipeArgs pa;
         pa.e = a;
@@ -935,9 +946,14 @@ cudaError_t encode_dispatch(const EncodeArgs& a, int codec, int norm, int scale,
 
 template <int CODEC, int NORM>
 cudaError_t decode_launch(const DecodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
-    static int per_tiles_grid = 0;
+    static PerDevice<int> cached;
     auto kern = decode_kernel<CODEC, NORM>;
-    if (per_tiles_grid == 0) per_tiles_grid = persistent_grid(kern, ~0ull >> 8, sm_count);
+    const int slot = device_slot();
+    int per_tiles_grid = slot >= 0 ? cached.v[slot] : 0;
+    if (per_tiles_grid == 0) {
+        per_tiles_grid = persistent_grid(kern, ~0ull >> 8, sm_count);
+        if (slot >= 0) cached.v[slot] = per_tiles_grid;
+    }
     const uint64_t want = (a.ntile - a.tile_begin + 7) / 8;
     const int grid = (int)(want < (uint64_t)per_tiles_grid ? (want ? want : 1) : (uint64_t)per_tiles_grid);
     kern<<<grid, kCodecThreads, 0, st>>>(a);

@@ -280,11 +280,12 @@ cudaError_t dots_cross(const DotsArgs& a, int grid, cudaStream_t st) {
 
 template <int NA>
 cudaError_t dots_pipe(const DotsPipeArgs& pa, int grid, cudaStream_t st) {
-    static bool configured = false;   // opt in to the large dynamic shared memory once per instantiation
-    if (!configured) {
+    static PerDevice<bool> configured;   // opt in to the large dynamic shared memory once per instantiation and device
+    const int slot = device_slot();
+    if (slot < 0 || !configured.v[slot]) {
         cudaError_t e = cudaFuncSetAttribute(dots_pipe_kernel<NA>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)DotsGeom::kSmemBytes);
         if (e != cudaSuccess) return e;
-        configured = true;
+        if (slot >= 0) configured.v[slot] = true;
     }
     dots_pipe_kernel<NA><<<grid, kDotsPipeThreads, DotsGeom::kSmemBytes, st>>>(pa);
     return cudaGetLastError();
@@ -328,47 +329,65 @@ cudaError_t dots_cross_n(int n, const DotsArgs& a, int grid, cudaStream_t st) {
 }
 
 // ---------------------------------------------------------------------------
-// K x K solve: one warp, lane 0 runs the Cholesky in double (k <= 16).
-// mode: TNG_FUSE_LSQ, TNG_FUSE_HINDSIGHT, TNG_FUSE_MEAN.
+// K x K ridge solve by one warp (k <= 16), fp64.  mode: TNG_FUSE_LSQ, TNG_FUSE_HINDSIGHT,
+// TNG_FUSE_MEAN, TNG_FUSE_LAST.
+//
+// Lane i owns row i of the augmented system [A | b] in shared memory.  Elimination is
+// right-looking: at step j every lane below the pivot scales its entry of column j by the
+// pivot's root, then subtracts the rank-one term from the rest of its row and from its b.
+// When the sweep ends column n holds the forward-substituted right-hand side, so only the
+// backward sweep (column by column, again one lane per row) remains.  A pivot that is not a
+// finite positive number above 1e-12 of the diagonal entry it started from is rounding
+// noise of a singular matrix: the solve reports failure and the caller falls back to the
+// newest history vector alone.
 // ---------------------------------------------------------------------------
-__device__ bool chol_solve(const double* A, const double* rhs, int n, double* x) {
-    double L[kMaxK * kMaxK];
-    double y[kMaxK];
+constexpr int kSolveLd = kMaxK + 1;   // row stride of the augmented system
+
+// S: n rows of n + 1 entries (stride kSolveLd); all 32 lanes call; returns the same verdict in every lane
+// and leaves the solution in x[0..n).
+__device__ bool warp_spd_solve(double* S, double* x, const int n, const int lane) {
+    const double start_diag = (lane < n) ? S[lane * kSolveLd + lane] : 1.0;
+    bool good = true;
     for (int j = 0; j < n; ++j) {
-        double diag = A[j * n + j];
-        for (int p = 0; p < j; ++p) diag -= L[j * n + p] * L[j * n + p];
-        // a pivot that is not above 1e-12 of its diagonal entry is rounding noise of a singular matrix
-        if (!(diag > 1e-12 * A[j * n + j]) || !(diag > 0.0) || !isfinite(diag)) return false;
-        const double ljj = sqrt(diag);
-        L[j * n + j] = ljj;
-        for (int i = j + 1; i < n; ++i) {
-            double v = A[i * n + j];
-            for (int p = 0; p < j; ++p) v -= L[i * n + p] * L[j * n + p];
-            L[i * n + j] = v / ljj;
+        const double piv = S[j * kSolveLd + j];
+        const double ref = __shfl_sync(kFullMask, start_diag, j);
+        if (!(piv > 1e-12 * ref) || !(piv > 0.0) || !isfinite(piv)) { good = false; break; }   // the same in all lanes
+        const double root = sqrt(piv);
+        __syncwarp();
+        if (lane >= j && lane < n) S[lane * kSolveLd + j] = (lane == j) ? root : S[lane * kSolveLd + j] / root;
+        if (lane == j) S[j * kSolveLd + n] /= root;
+        __syncwarp();
+        if (lane > j && lane < n) {
+            const double mine = S[lane * kSolveLd + j];
+            for (int c = j + 1; c <= lane; ++c) S[lane * kSolveLd + c] -= mine * S[c * kSolveLd + j];
+            S[lane * kSolveLd + n] -= mine * S[j * kSolveLd + n];
         }
+        __syncwarp();
     }
-    for (int i = 0; i < n; ++i) {
-        double v = rhs[i];
-        for (int p = 0; p < i; ++p) v -= L[i * n + p] * y[p];
-        y[i] = v / L[i * n + i];
-    }
+    if (!good) return false;
+    // backward sweep on L^T: the newest unknown is final, every lane above it removes its share
     for (int i = n - 1; i >= 0; --i) {
-        double v = y[i];
-        for (int p = i + 1; p < n; ++p) v -= L[p * n + i] * x[p];
-        x[i] = v / L[i * n + i];
+        if (lane == i) S[i * kSolveLd + n] /= S[i * kSolveLd + i];
+        __syncwarp();
+        if (lane < i) S[lane * kSolveLd + n] -= S[i * kSolveLd + lane] * S[i * kSolveLd + n];
+        __syncwarp();
     }
-    for (int i = 0; i < n; ++i)
-        if (!isfinite(x[i])) return false;
-    return true;
+    const double xi = (lane < n) ? S[lane * kSolveLd + n] : 0.0;
+    if (lane < n) x[lane] = xi;
+    __syncwarp();
+    return __all_sync(kFullMask, isfinite(xi));
 }
 
 __global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mode, double ridge, int have_rhs, double rhs_div) {
     // the whole warp brings the statistics into shared memory (one round trip to global memory
-    // instead of one per entry); lane 0 then works on the copy and writes the mirrored Gram back
+    // instead of one per entry) and writes the mirrored Gram back
     __shared__ double sG[kGramDoubles];
+    __shared__ double sS[kMaxK * kSolveLd];
+    __shared__ double sx[kMaxK];
+    const int lane = threadIdx.x;
     const bool stats = (mode == TNG_FUSE_LSQ) || (mode == TNG_FUSE_HINDSIGHT);
-    if (stats)
-        for (int i = threadIdx.x; i < kGramDoubles; i += 32) {
+    if (stats) {
+        for (int i = lane; i < kGramDoubles; i += 32) {
             double v = fb->gram[i];
             if (rhs_div != 1.0 && i >= kGramRhs) {   // sums over all workers -> means
                 v /= rhs_div;
@@ -376,76 +395,76 @@ __global__ void __launch_bounds__(32) solve_kernel(FuseBlock* fb, int k, int mod
             }
             sG[i] = v;
         }
-    __syncwarp();
-    if (threadIdx.x != 0) return;
-    double alpha[kMaxK];
-    for (int j = 0; j < kMaxK; ++j) alpha[j] = 0.0;
+        __syncwarp();
+        for (int i = lane; i < k * k; i += 32) {   // mirror the upper triangle
+            const int a = i / k, b = i % k;
+            if (b < a) {
+                const double v = sG[b * kGramStride + a];
+                sG[a * kGramStride + b] = v;
+                fb->gram[a * kGramStride + b] = v;
+            }
+        }
+        __syncwarp();
+    }
+    double alpha = 0.0;   // lane j holds alpha_j
     uint32_t fallback = 0;
-    double* G = sG;
     if (mode == TNG_FUSE_MEAN) {
-        const float inv = __fdiv_rn(1.0f, (float)k);
-        for (int j = 0; j < k; ++j) alpha[j] = (double)inv;
+        if (lane < k) alpha = (double)__fdiv_rn(1.0f, (float)k);
     } else if (mode == TNG_FUSE_LAST) {
-        alpha[0] = 1.0;
+        if (lane == 0) alpha = 1.0;
     } else {
-        for (int a = 0; a < k; ++a)   // mirror the upper triangle
-            for (int b = 0; b < a; ++b) fb->gram[a * kGramStride + b] = G[a * kGramStride + b] = G[b * kGramStride + a];
-        double A[kMaxK * kMaxK], rhs[kMaxK], x[kMaxK];
-        bool ok;
-        if (mode == TNG_FUSE_LSQ) {
+        // LSQ: all k vectors against <h_j, mean gradient>.  Hindsight: regress h_1 on h_2..h_k (the
+        // sub-Gram without row/column 0 against column 0) and apply the coefficients one position later.
+        const int off = (mode == TNG_FUSE_LSQ) ? 0 : 1;
+        const int n = k - off;
+        if (n >= 1) {
+            double tr = (lane < n) ? sG[(lane + off) * kGramStride + lane + off] : 0.0;
+            // the trace is summed serially, entry 0 first (the order of a plain loop)
             double trace = 0.0;
-            for (int j = 0; j < k; ++j) trace += G[j * kGramStride + j];
-            const double lambda = ridge * trace / (double)k;
-            for (int a = 0; a < k; ++a) {
-                rhs[a] = G[kGramRhs + a];
-                for (int b = 0; b < k; ++b) A[a * k + b] = G[a * kGramStride + b] + (a == b ? lambda : 0.0);
+            for (int j = 0; j < n; ++j) trace += __shfl_sync(kFullMask, tr, j);
+            const double lambda = ridge * trace / (double)n;
+            if (lane < n) {
+                for (int b = 0; b < n; ++b) sS[lane * kSolveLd + b] = sG[(lane + off) * kGramStride + b + off] + (b == lane ? lambda : 0.0);
+                sS[lane * kSolveLd + n] = (mode == TNG_FUSE_LSQ) ? sG[kGramRhs + lane] : sG[(lane + 1) * kGramStride];
             }
-            ok = chol_solve(A, rhs, k, x);
-            if (ok) for (int j = 0; j < k; ++j) alpha[j] = x[j];
-        } else {   // hindsight: regress h_1 on h_2..h_k, apply one position later
-            const int n = k - 1;
-            ok = true;
-            if (n >= 1) {
-                double trace = 0.0;
-                for (int j = 1; j < k; ++j) trace += G[j * kGramStride + j];
-                const double lambda = ridge * trace / (double)n;
-                for (int a = 0; a < n; ++a) {
-                    rhs[a] = G[(a + 1) * kGramStride + 0];
-                    for (int b = 0; b < n; ++b)
-                        A[a * n + b] = G[(a + 1) * kGramStride + (b + 1)] + (a == b ? lambda : 0.0);
-                }
-                ok = chol_solve(A, rhs, n, x);
-                if (ok) for (int j = 0; j < n; ++j) alpha[j] = x[j];
+            __syncwarp();
+            if (warp_spd_solve(sS, sx, n, lane)) {
+                if (lane < n) alpha = sx[lane];
             } else {
-                alpha[0] = 1.0;
+                fallback = 1;
+                alpha = (lane == 0) ? 1.0 : 0.0;
             }
-        }
-        if (!ok) {
-            fallback = 1;
-            for (int j = 0; j < kMaxK; ++j) alpha[j] = 0.0;
-            alpha[0] = 1.0;
+        } else {
+            alpha = (lane == 0) ? 1.0 : 0.0;   // a single stored vector has no past to regress on
         }
     }
-    double a32[kMaxK];
-    for (int j = 0; j < kMaxK; ++j) {
-        fb->alpha64[j] = alpha[j];
-        const float f = (float)alpha[j];
-        fb->alpha32[j] = f;
-        a32[j] = (double)f;
+    const float a32f = (float)alpha;
+    if (lane < kMaxK) {
+        fb->alpha64[lane] = alpha;
+        fb->alpha32[lane] = a32f;
     }
-    fb->fallback = fallback;
-    // C_nz estimate from the statistics: (gg - 2 a.c + a^T G a) / gg with the fp32 coefficients
+    if (lane == 0) fb->fallback = fallback;
+    // C_nz estimate from the statistics: (gg - 2 a.c + a^T G a) / gg with the fp32 coefficients;
+    // lane a takes row a, the rows are added in lane order
     double cnz = nan("");
     if (have_rhs && mode != TNG_FUSE_MEAN) {
+        const double a32 = (double)a32f;
+        double row = 0.0;
+        for (int b = 0; b < k; ++b) {
+            const double ab = __shfl_sync(kFullMask, a32, b);
+            if (lane < k) row += ab * sG[lane * kGramStride + b];
+        }
+        double quad_l = (lane < k) ? a32 * row : 0.0;
+        double lin_l = (lane < k) ? a32 * sG[kGramRhs + lane] : 0.0;
         double quad = 0.0, lin = 0.0;
         for (int a = 0; a < k; ++a) {
-            lin += a32[a] * G[kGramRhs + a];
-            for (int b = 0; b < k; ++b) quad += a32[a] * a32[b] * G[a * kGramStride + b];
+            quad += __shfl_sync(kFullMask, quad_l, a);
+            lin += __shfl_sync(kFullMask, lin_l, a);
         }
-        const double gg = G[kGramGG];
+        const double gg = sG[kGramGG];
         cnz = (gg - 2.0 * lin + quad) / gg;
     }
-    fb->cnz = cnz;
+    if (lane == 0) fb->cnz = cnz;
 }
 
 // ---------------------------------------------------------------------------
@@ -504,7 +523,9 @@ cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float
     const uint64_t ngroups = (d + 3) / 4;
     uint64_t want = (ngroups + kDotsThreads - 1) / kDotsThreads;
     if (want < 1) want = 1;
-    const int grid = (int)(want < (uint64_t)sm_count ? want : (uint64_t)sm_count);
+    // one partial row per CTA: never more CTAs than the partials buffer has rows
+    const uint64_t max_ctas = (uint64_t)(sm_count < kDotsMaxCtas ? sm_count : kDotsMaxCtas);
+    const int grid = (int)(want < max_ctas ? want : max_ctas);
     DotsArgs a;
     a.grads = grads; a.partials = partials; a.fb = fb; a.d = d; a.ld = ld; a.M = M;
     a.divisor = divisor ? divisor : M;
@@ -525,7 +546,7 @@ cudaError_t launch_dots(const float* const* rows, int k, uint64_t d, const float
         if (grads)
             for (uint32_t m = 0; m < M; ++m) pa.rows.row[pa.rows.nrows++] = grads + (uint64_t)m * ld;
         const uint64_t nchunks = d / DotsGeom::kChunk;
-        const int pgrid = (int)(nchunks < (uint64_t)sm_count ? nchunks : (uint64_t)sm_count);
+        const int pgrid = (int)(nchunks < max_ctas ? nchunks : max_ctas);
         e = dots_pipe_n(k, pa, pgrid, st);
         ++*launches;
         return e;

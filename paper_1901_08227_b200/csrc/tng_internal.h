@@ -16,6 +16,20 @@ constexpr int kGramDoubles = kGramGG + 1;
 constexpr int kDotsMaxAcc = 64;                         // accumulators of one dots launch
 constexpr int kDotsMaxCtas = 592;                       // 4 x 148
 
+// Function attributes (the dynamic shared-memory opt-in) and occupancy belong to a device, not
+// to the process: a value cached per kernel instantiation is kept per device index.  Devices
+// beyond the table are simply not cached (slot() < 0: the caller sets / asks every time).
+constexpr int kMaxDevices = 64;
+inline int device_slot() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return -1;
+    return dev;
+}
+template <typename T>
+struct PerDevice {
+    T v[kMaxDevices] = {};
+};
+
 // Small device-resident block: fusion statistics, coefficients, flags.
 struct FuseBlock {
     double gram[kGramDoubles + 7];   // padded to 280 doubles

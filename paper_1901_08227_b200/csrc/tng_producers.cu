@@ -177,11 +177,26 @@ __global__ void __launch_bounds__(256) sgd_update_kernel(float* __restrict__ w, 
 // Row chunks of the transposed product: enough CTAs to fill the GPU (4 per SM), and, when a
 // count up to the limit exists, a total that is a multiple of the SM count so that no SM gets
 // one CTA more than another.
+// SM count of the current device (asked once per device index).
+int sm_count_now() {
+    static PerDevice<int> cached;
+    const int slot = device_slot();
+    if (slot >= 0 && cached.v[slot] > 0) return cached.v[slot];
+    int dev = 0, sms = 0;
+    if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || sms < 1) {
+        (void)cudaGetLastError();
+        sms = 1;
+    }
+    if (slot >= 0) cached.v[slot] = sms;
+    return sms;
+}
+
 int row_chunks(uint64_t n, uint64_t d, bool vec) {
     const uint64_t colblocks = ((vec ? d / 4 : d) + 255) / 256;
-    uint64_t chunks = (592 + colblocks - 1) / colblocks;
+    const uint64_t sms = (uint64_t)sm_count_now();
+    uint64_t chunks = (4 * sms + colblocks - 1) / colblocks;
     for (uint64_t c = chunks; c <= (uint64_t)kMaxRowChunks; ++c)
-        if ((colblocks * c) % 148 == 0) { chunks = c; break; }
+        if ((colblocks * c) % sms == 0) { chunks = c; break; }
     if (chunks > (uint64_t)kMaxRowChunks) chunks = kMaxRowChunks;
     if (chunks > n) chunks = n;
     if (chunks < 1) chunks = 1;
@@ -194,7 +209,8 @@ bool vec_ok(const float* X, const float* w, uint64_t d) {
 
 cudaError_t launch_margins(const float* X, const float* b, const float* w, uint64_t n, uint64_t d, float* coef,
                            float* lossrow, cudaStream_t st) {
-    const int grid = (int)(n < 148 * 64 ? n : 148 * 64);
+    const uint64_t cap = (uint64_t)sm_count_now() * 64u;
+    const int grid = (int)(n < cap ? n : cap);
     if (vec_ok(X, w, d)) logistic_margin_kernel<true><<<grid, 256, 0, st>>>(X, b, w, n, d, coef, lossrow);
     else logistic_margin_kernel<false><<<grid, 256, 0, st>>>(X, b, w, n, d, coef, lossrow);
     return cudaGetLastError();
@@ -255,7 +271,8 @@ tng_status tng_rosenbrock_grad(const float* x_dev, uint64_t d, const float* nois
         return TNG_ERR_INVALID_ARG;
     const uint64_t npairs = d / 2;
     const uint64_t want = (npairs + 255) / 256;
-    const int grid = (int)(want < 2368 ? want : 2368);
+    const uint64_t cap = (uint64_t)sm_count_now() * 16u;
+    const int grid = (int)(want < cap ? want : cap);
     rosenbrock_grad_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(x_dev, npairs, noise_dev, M, ld, grads_dev);
     return cudaGetLastError() == cudaSuccess ? TNG_OK : TNG_ERR_CUDA;
 }
@@ -269,7 +286,8 @@ tng_status tng_rosenbrock_value(const float* x_dev, uint64_t d, double* value_de
 tng_status tng_sgd_update(float* w_dev, const float* v_dev, uint64_t d, float eta, void* stream) {
     if (!w_dev || !v_dev || d < 1) return TNG_ERR_INVALID_ARG;
     const uint64_t want = (d + 255) / 256;
-    const int grid = (int)(want < 2368 ? want : 2368);
+    const uint64_t cap = (uint64_t)sm_count_now() * 16u;
+    const int grid = (int)(want < cap ? want : cap);
     sgd_update_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(w_dev, v_dev, d, eta);
     return cudaGetLastError() == cudaSuccess ? TNG_OK : TNG_ERR_CUDA;
 }

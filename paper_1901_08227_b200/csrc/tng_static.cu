@@ -26,18 +26,24 @@ static_assert(kTngStaticScratchBytes <= TNG_STATIC_SCRATCH_BYTES, "header states
 // for the symbol.  The device address comes from cudaGetSymbolAddress (below).
 static __device__ __align__(256) unsigned char g_static_scratch[TNG_STATIC_SCRATCH_BYTES];
 
-constexpr int kMaxDevices = 64;
+using tng::kMaxDevices;
 void* g_scratch_addr[kMaxDevices] = {nullptr};   // per device, filled on first use
 int g_sm_count[kMaxDevices] = {0};
 
 // Packs the statistics from the scratch block into the caller's buffer:
 // out[0 .. k*k) = G row-major (both triangles), out[k*k .. k*k+k) = rhs, out[k*k+k] = grad_sq.
+// If a bounded wait of the staged statistics kernel gave up, the sums are incomplete: every
+// output becomes NaN, which is how this entry point (it never synchronises with the host)
+// reports that.
 __global__ void pack_static_gram_kernel(int k, double* __restrict__ out) {
     const FuseBlock* fb = reinterpret_cast<const FuseBlock*>(g_static_scratch + kBlockOffset);   // device code may name the array
     const int n = k * k + k + 1;
+    const bool gave_up = fb->pipe_error != 0u;
     for (int i = threadIdx.x; i < n; i += blockDim.x) {
         double v;
-        if (i < k * k) {
+        if (gave_up) {
+            v = nan("");
+        } else if (i < k * k) {
             const int a = i / k, b = i % k;
             v = (a <= b) ? fb->gram[a * tng::kGramStride + b] : fb->gram[b * tng::kGramStride + a];
         } else if (i < k * k + k) {

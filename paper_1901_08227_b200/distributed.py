@@ -39,7 +39,12 @@ class DistributedRound:
         self.world = dist.get_world_size(group) if group is not None else 1
         self.rank = dist.get_rank(group) if group is not None else 0
         self.first, self.count = worker_range(self.rank, self.world, ctx.M)
-        self.round = 0
+        self.resync()
+
+    def resync(self):
+        """Take the round number (the Philox step) from the context: it is ahead of zero after a
+        loaded state or earlier rounds, and the codes must use the context's own counter."""
+        self.round = int(self.ctx.stats().rounds)
 
     def step(self, local_grads: torch.Tensor, out: torch.Tensor | None = None):
         """local_grads: (count, d) rows of this rank's workers.  Returns `out` (the aggregate)."""
@@ -94,7 +99,11 @@ class CoordShardedRound:
     def __init__(self, ctx: tng.Context, group=None):
         self.ctx, self.group = ctx, group
         self.world = dist.get_world_size(group) if group is not None else 1
-        self.round = 0
+        self.resync()
+
+    def resync(self):
+        """Take the round number (the Philox step) from the context, see DistributedRound.resync."""
+        self.round = int(self.ctx.stats().rounds)
 
     def step(self, grads_slice: torch.Tensor, out: torch.Tensor | None = None):
         """grads_slice: (M, count) — this rank's coordinates of every worker's gradient."""

@@ -87,8 +87,9 @@ def test_long_vectors_take_the_staged_kernels(codec, norm, scale_kind, M, d):
 
 
 @pytest.mark.parametrize("codec", CODECS)
+@pytest.mark.parametrize("scale_kind", [0, 1])
 @pytest.mark.parametrize("factor", [1e-28, 1e-33, 1e-38, 3e-42])
-def test_tiny_and_subnormal_scales(codec, factor):
+def test_tiny_and_subnormal_scales(codec, factor, scale_kind):
     # scales around and below 2^-100 (and subnormal ones): the rounding threshold u*R must be the
     # same correctly rounded product on both sides
     d, M = 2048 * 9 + 128 * 3 + 50, 4
@@ -96,16 +97,40 @@ def test_tiny_and_subnormal_scales(codec, factor):
     g.mul_(factor)
     g[1, 128 * 5: 128 * 6] *= 1e6                       # one ordinary-looking block among the tiny ones
     ref = (g.mean(0) * 0.5).contiguous()
-    ctx = make_ctx(d, M, 1, codec, tng.NORM_DIFF, block=128, seed_lo=1)
+    ctx = make_ctx(d, M, 1, codec, tng.NORM_DIFF, block=128, seed_lo=1, scale_kind=scale_kind)
     ctx.encode(g, ref=ref, step=3)
     codes, scales = ctx.wire()
     out = torch.empty(d, device="cuda")
     ctx.decode_aggregate(out, ref=ref)
     gn, rn = to_np(g), to_np(ref)
-    oc, osc = oracle.encode(gn, rn, tng.NORM_DIFF, codec, B=128, s=7, seed=(1, 0), t=3)
+    oc, osc = oracle.encode(gn, rn, tng.NORM_DIFF, codec, B=128, s=7, seed=(1, 0), t=3, scale_kind=scale_kind)
     assert same_values(to_np(scales), osc) and np.array_equal(codes_np(codes), oc)
     assert np.array_equal(to_np(out).view(np.uint32), oracle.decode_aggregate(oc, osc, d, rn, tng.NORM_DIFF, codec, B=128, s=7).view(np.uint32))
-    assert oc.any()
+    # (with the L2 scale every square underflows below ~1e-23: all scales and all codes are zero then)
+    assert oc.any() or (scale_kind == 1 and factor < 1e-28)
+
+
+@pytest.mark.parametrize("d", [128 * 4, 2048 * 9 + 128 * 3 + 50])
+def test_quantiser_level_is_bounded_when_the_l2_scale_falls_short(d):
+    # blocks whose only non-zero element has a subnormal square: sqrt(fl(v*v)) < |v|, so s|v|/R > s; the level
+    # must stay s and the sign plane must hold the sign (both the direct and the staged kernel)
+    M, s = 4, 7
+    g = torch.zeros(M, round_up4(d), device="cuda")
+    for T in range(0, d // 128, 3):
+        g[:, 128 * T + (37 * T) % 128] = torch.tensor([1e-22, 3e-22, -1e-22, -3e-22], device="cuda")
+    g[2, 128: 256] = workloads.normal((128,), 5, 2, "cuda")          # an ordinary block among them
+    for step in range(6):
+        ctx = make_ctx(d, M, 1, tng.CODEC_QSGD4, tng.NORM_NONE, block=128, seed_lo=2, scale_kind=1, qsgd_levels=s)
+        ctx.encode(g, step=step)
+        codes, scales = ctx.wire()
+        out = torch.empty(d, device="cuda")
+        ctx.decode_aggregate(out)
+        gn = to_np(g)[:, :d]
+        oc, osc = oracle.encode(gn, None, tng.NORM_NONE, tng.CODEC_QSGD4, B=128, s=s, seed=(2, 0), t=step, scale_kind=1)
+        assert same_values(to_np(scales), osc) and np.array_equal(codes_np(codes), oc)
+        want = oracle.decode_aggregate(oc, osc, d, None, tng.NORM_NONE, tng.CODEC_QSGD4, B=128, s=s)
+        assert np.array_equal(to_np(out).view(np.uint32), want.view(np.uint32))
+        ctx.close()
 
 
 @pytest.mark.parametrize("s", [1, 2, 3, 4, 5, 6, 7])

@@ -121,6 +121,11 @@ class _OracleSliceContext:
         self.block = torch.zeros(273, dtype=torch.float64)
         self.ref = np.zeros(count, dtype=np.float32)
         self.alpha = np.zeros(K, dtype=np.float32)
+        self.rounds = 0
+
+    def stats(self):
+        from types import SimpleNamespace
+        return SimpleNamespace(rounds=self.rounds)
 
     def fuse_local(self, g):
         self.block.zero_()
@@ -160,6 +165,7 @@ class _OracleSliceContext:
         codes, scales = self.wire
         res = self.o.decode_aggregate(codes, scales, self.d, self.ref, self.norm, self.codec, B=128)
         self.hist = ([res] + self.hist)[:self.K]
+        self.rounds += 1
         if out is not None:
             out.copy_(torch.from_numpy(res))
 
@@ -177,6 +183,9 @@ def _sliced_main(rank, world, port, out_dir, mode):
     outs, alphas = [], []
     mean = rng.standard_normal(d).astype(np.float32)
     for t in range(steps):
+        if t == 3:   # a driver created in mid-run takes the round number (the Philox step) from the context
+            drv = distributed.CoordShardedRound(ctx, group=dist.group.WORLD)
+            assert drv.round == 3
         mean = (0.9 * mean + 0.3 * rng.standard_normal(d)).astype(np.float32)
         g = (mean[None] + 0.5 * rng.standard_normal((M, d))).astype(np.float32)
         out = torch.empty(count)

@@ -9,6 +9,7 @@ import numpy as np
 import pytest
 import torch
 
+import oracle
 from paper_1901_08227_b200 import tng, workloads
 
 pytestmark = pytest.mark.gpu
@@ -45,6 +46,13 @@ def test_static_scratch_path_matches_the_context_path_twice_in_a_row(k, M, d):
         assert np.abs(got - want).max() <= 1e-10 * scale, f"call {call}"
         G = got[: k * k].reshape(k, k)
         assert np.array_equal(G, G.T)
+        # and against the CPU oracle's double-precision sums, so that this test stands on its own
+        oG, oc, ogg = oracle.fuse_stats([r.cpu().numpy() for r in rows], grads.cpu().numpy()[:, :d])
+        owant = np.concatenate([oG.ravel(), oc, [ogg]])
+        # (the Gram sums are double throughout; the gradient sums over the M workers are formed in fp32
+        # per coordinate before they enter the double accumulators, hence the looser bound on rhs and norm)
+        assert np.abs(got[: k * k] - owant[: k * k]).max() <= 1e-10 * np.abs(owant[: k * k]).max(), f"call {call} (oracle, Gram)"
+        assert np.abs(got[k * k:] - owant[k * k:]).max() <= 1e-6 * np.abs(owant[k * k:]).max(), f"call {call} (oracle, rhs)"
 
 
 def test_sizes_beyond_the_fixed_scratch_are_rejected():
