@@ -475,6 +475,159 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
     }
 }
 
+// ---------------------------------------------------------------------------
+// The same pass when one scale spans 2, 4, 8 or 16 tiles (blocks of 256 .. 2048
+// coordinates, all inside one chunk): the gradient rows are still read once.  Per fill a
+// warp normalises its tile for the (up to) eight workers, keeps the values in registers and
+// posts the eight tile statistics in shared memory; after a barrier among the compute warps,
+// lane k of every warp combines the statistics of its block for worker k (maximum, or the
+// adjacent-pairwise sum that continues the tree inside the tiles; slots beyond the block count
+// as zero, the identity of both) and the warp quantises from registers.  Statistics and the
+// give-up flag are double-buffered, so one barrier per fill is enough: a warp can only run one
+// fill ahead of the slowest one.  A warp whose bounded wait runs out raises the flag and still
+// arrives at the fill's barrier; after it all sixteen warps see the flag and leave together,
+// so nobody is left waiting at a barrier.
+// ---------------------------------------------------------------------------
+__device__ __forceinline__ void compute_warps_barrier() {
+    asm volatile("bar.sync 1, %0;" ::"n"(kEncPipeWarps * 32) : "memory");
+}
+
+template <int CODEC, int NORM, int SCALE, bool FUSEREF>
+__global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_blocks_kernel(const EncodePipeArgs pa) {
+    using G = EncGeom;
+    extern __shared__ unsigned char dyn_smem[];
+    __shared__ float s_alpha[kMaxK];
+    __shared__ float s_stat[2][G::kRows][kEncPipeWarps + 1];
+    __shared__ uint32_t s_gave_up[2];
+    const EncodeArgs& a = pa.e;
+    if (FUSEREF && threadIdx.x < kMaxK) s_alpha[threadIdx.x] = ((int)threadIdx.x < a.hist_k) ? a.alpha[threadIdx.x] : 0.0f;
+    if (threadIdx.x < 2) s_gave_up[threadIdx.x] = 0u;
+    const PipeSmem pipe = pipe_setup<G>(dyn_smem, kEncPipeWarps);   // ends with __syncthreads
+    const uint64_t nchunks = a.tile_begin / kEncPipeWarps;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    if (warp == kEncPipeWarps) {
+        if (lane == 0) {
+            const uint32_t err = pipe_produce<G>(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
+            if (err != kPipeOk) atomicMax(a.pipe_error, err);
+        }
+        return;
+    }
+    const uint32_t my = (uint32_t)warp * (kTile * 4u) + (uint32_t)lane * 16u;
+    const unsigned char* stages = dyn_smem + (pipe.data - smem_u32(dyn_smem));
+    const int n_pre = pa.rows.n_pre;
+    const uint32_t M = a.M;
+    const int tpb = (int)(a.block / kTile);                // tiles per block: 2, 4, 8 or 16
+    const int block_warp0 = warp & ~(tpb - 1);             // first warp (tile) of this warp's block within the chunk
+    constexpr int kWords = 4 * CODEC;
+    uint32_t it = 0, buf = 0;
+    bool alive = true;
+    for (uint64_t c = blockIdx.x; c < nchunks; c += gridDim.x) {
+        const uint64_t T = c * kEncPipeWarps + (uint32_t)warp;
+        const uint64_t blk = T / (uint32_t)tpb;
+        const uint64_t q = (T + a.tile0) * 32u + (uint32_t)lane;
+        const uint32_t q_lo = (uint32_t)q, q_hi = (uint32_t)(q >> 32);
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
+        for (int p0 = 0; p0 < n_pre && alive; p0 += G::kRows) {
+            const int n = (n_pre - p0 < G::kRows) ? n_pre - p0 : G::kRows;
+            const uint32_t s = it % G::kStages, use = it / G::kStages;
+            if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {
+                atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
+                s_gave_up[buf] = 1u;
+                alive = false;
+                break;
+            }
+            const unsigned char* base = stages + s * G::kStageBytes + my;
+            if (FUSEREF) {
+                for (int j = 0; j < n; ++j) {
+                    const float4 x = *reinterpret_cast<const float4*>(base + (uint32_t)j * G::kRowBytes);
+                    const float al = s_alpha[p0 + j];
+                    r.x = __fmaf_rn(al, x.x, r.x); r.y = __fmaf_rn(al, x.y, r.y);
+                    r.z = __fmaf_rn(al, x.z, r.z); r.w = __fmaf_rn(al, x.w, r.w);
+                    if (NORM == TNG_NORM_COMB) magnitude_fma(r2, a.inv_k, x);
+                }
+            } else {
+                r = *reinterpret_cast<const float4*>(base);
+                if (NORM == TNG_NORM_COMB && n > 1) r2 = *reinterpret_cast<const float4*>(base + G::kRowBytes);
+            }
+            __syncwarp();
+            if (lane == 0) mbar_arrive(pipe.empty(s));
+            ++it;
+        }
+        if (FUSEREF && alive) {
+            *reinterpret_cast<float4*>(a.ref_out + (T * kTile + (uint64_t)lane * 4u)) = r;
+            if (NORM == TNG_NORM_COMB) *reinterpret_cast<float4*>(a.ref2_out + (T * kTile + (uint64_t)lane * 4u)) = r2;
+        }
+        const NormOp op = make_norm_op<NORM>(r, r2, a.quot_eps);
+        for (uint32_t m0 = 0; m0 < M; m0 += G::kRows) {
+            float v[G::kRows][4];
+            float my_stat = 0.0f;
+            if (alive) {
+                const uint32_t s = it % G::kStages, use = it / G::kStages;
+                if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {
+                    atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
+                    s_gave_up[buf] = 1u;
+                    alive = false;
+                }
+                if (alive) {
+                    const unsigned char* base = stages + s * G::kStageBytes + my;
+#pragma unroll
+                    for (int k = 0; k < G::kRows; ++k) {
+                        if (m0 + k < M) {   // the same answer in every thread of the grid
+                            const float4 g = *reinterpret_cast<const float4*>(base + (uint32_t)k * G::kRowBytes);
+                            encode_normalise<NORM>(g, worker_op<NORM>(a, op, m0 + k), v[k]);
+                            const float st = encode_tile_stat<SCALE>(v[k]);
+                            my_stat = (lane == k) ? st : my_stat;
+                        }
+                    }
+                    __syncwarp();
+                    if (lane == 0) mbar_arrive(pipe.empty(s));
+                    ++it;
+                    if (lane < G::kRows) s_stat[buf][lane][warp] = my_stat;
+                }
+            }
+            compute_warps_barrier();
+            if (s_gave_up[buf] != 0u) return;              // the same answer in all sixteen warps
+            // lane k: the block's statistic for worker k of the fill
+            float bs[kEncPipeWarps];
+#pragma unroll
+            for (int t = 0; t < kEncPipeWarps; ++t) bs[t] = (t < tpb) ? s_stat[buf][lane & (G::kRows - 1)][block_warp0 + t] : 0.0f;
+#pragma unroll
+            for (int len = kEncPipeWarps; len > 1; len >>= 1)
+#pragma unroll
+                for (int t = 0; t < len / 2; ++t)
+                    bs[t] = (SCALE == 0) ? __uint_as_float(max(__float_as_uint(bs[2 * t]), __float_as_uint(bs[2 * t + 1])))
+                                         : __fadd_rn(bs[2 * t], bs[2 * t + 1]);
+            const float my_R = (SCALE == 0) ? bs[0] : __fsqrt_rn(bs[0]);
+            const uint32_t mine = m0 + (uint32_t)lane;
+            uint32_t* my_codes = a.codes + ((uint64_t)mine * a.wpw + T * (uint64_t)kWords);
+#pragma unroll
+            for (int k0 = 0; k0 < G::kRows; k0 += kPhiloxBatch) {
+                if (m0 + k0 < M) {
+                    uint4 x[kPhiloxBatch];
+                    philox4x32_10_rk_batch<kPhiloxBatch>(q_lo, q_hi, a.m_base + m0 + k0, a.step, a.rk, x);
+#pragma unroll
+                    for (int kk = 0; kk < kPhiloxBatch; ++kk) {
+                        const int k = k0 + kk;
+                        if (m0 + k < M) {
+                            const float R = __shfl_sync(kFullMask, my_R, k);
+                            const float Rq = (SCALE == 1 && !(R > 0.0f)) ? __int_as_float(0x7fc00000) : R;
+                            uint32_t w[kWords];
+                            encode_quantise<CODEC, true>(a, v[k], Rq, x[kk], 0xFu, w);
+                            store_words_if<CODEC>(lane == k, my_codes, w);
+                        }
+                    }
+                }
+            }
+            // the first warp of a block writes its scales
+            const bool writes = warp == block_warp0 && lane < G::kRows && mine < M;
+            if (writes) a.scales[(uint64_t)mine * a.nblk + blk] = my_R;
+            const uint32_t bad = __ballot_sync(kFullMask, writes && __float_as_uint(my_R) >= 0x7f800000u);
+            if (bad != 0u && lane == 0) atomicAdd(a.nonfinite, (unsigned long long)__popc(bad));
+            buf ^= 1u;
+        }
+    }
+}
+
 // Scalar reference (Section 3.1), first pass: the sum of every tile of every row, as the
 // adjacent-pairwise fp32 tree (the lane's four values pairwise, then xor-shuffles pair
 // neighbouring lanes); elements past the end count as zero.  The tree over the tiles and
@@ -503,19 +656,12 @@ __global__ void __launch_bounds__(kCodecThreads) row_tile_sum_kernel(const float
 // SCALE 2 is the plain sum behind the scalar reference: its last level divides by `divisor`
 // (the vector length) and the value becomes the worker's mean.
 constexpr int kTreeSum = 2;
+
+// The tree over 1024 shared-memory entries (256 threads, all of them call): adjacent pairs level by
+// level, a sum (SCALE 1, 2) or the maximum of the bit patterns (SCALE 0: non-negative floats and NaNs
+// order like their patterns).  The result is left in buf[0], visible to every thread.
 template <int SCALE>
-__global__ void __launch_bounds__(256) block_scale_level_kernel(const float* __restrict__ in, uint64_t n_in,
-                                                                uint64_t seg, uint64_t chunks_per_seg,
-                                                                float* __restrict__ out, uint64_t n_out,
-                                                                int final, float divisor, unsigned long long* nonfinite) {
-    __shared__ float buf[1024];
-    const uint64_t s = blockIdx.x, c = blockIdx.y, m = blockIdx.z;
-    const uint64_t seg_lo = s * seg;
-    const uint64_t seg_hi = (seg_lo + seg < n_in) ? seg_lo + seg : n_in;
-    const uint64_t lo = seg_lo + c * 1024u;
-    const float* row = in + m * n_in;
-    for (int i = threadIdx.x; i < 1024; i += 256) buf[i] = (lo + i < seg_hi) ? row[lo + i] : 0.0f;
-    __syncthreads();
+__device__ __forceinline__ void cta_tree_1024(float* buf) {
     for (int len = 1024; len > 1; len >>= 1) {
         float t0 = 0.f, t1 = 0.f;
         const int i0 = threadIdx.x, i1 = threadIdx.x + 256;
@@ -532,6 +678,22 @@ __global__ void __launch_bounds__(256) block_scale_level_kernel(const float* __r
         if (i1 < len / 2) buf[i1] = t1;
         __syncthreads();
     }
+}
+
+template <int SCALE>
+__global__ void __launch_bounds__(256) block_scale_level_kernel(const float* __restrict__ in, uint64_t n_in,
+                                                                uint64_t seg, uint64_t chunks_per_seg,
+                                                                float* __restrict__ out, uint64_t n_out,
+                                                                int final, float divisor, unsigned long long* nonfinite) {
+    __shared__ float buf[1024];
+    const uint64_t s = blockIdx.x, c = blockIdx.y, m = blockIdx.z;
+    const uint64_t seg_lo = s * seg;
+    const uint64_t seg_hi = (seg_lo + seg < n_in) ? seg_lo + seg : n_in;
+    const uint64_t lo = seg_lo + c * 1024u;
+    const float* row = in + m * n_in;
+    for (int i = threadIdx.x; i < 1024; i += 256) buf[i] = (lo + i < seg_hi) ? row[lo + i] : 0.0f;
+    __syncthreads();
+    cta_tree_1024<SCALE>(buf);
     if (threadIdx.x == 0) {
         float r = buf[0];
         if (final) {
@@ -540,6 +702,101 @@ __global__ void __launch_bounds__(256) block_scale_level_kernel(const float* __r
             if (!(fabsf(r) < __int_as_float(0x7f800000))) atomicAdd(nonfinite, 1ull);
         }
         out[m * n_out + s * chunks_per_seg + c] = r;
+    }
+}
+
+// ---------------------------------------------------------------------------
+// Short problems (a per-vector scale at small d, odd block sizes of short vectors): the three
+// launches statistic -> tree -> quantise are latency, not bandwidth.  Here one CTA owns one
+// scale block of one worker (at most 1024 tiles): its warps compute the tile statistics into
+// shared memory, the CTA runs the same tree as block_scale_level_kernel, and the warps go over
+// the tiles again (now cache-resident) to quantise.  One launch.
+// ---------------------------------------------------------------------------
+template <int CODEC, int NORM, int SCALE>
+__global__ void __launch_bounds__(256) encode_block_cta_kernel(const EncodeArgs a) {
+    __shared__ float buf[1024];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const uint32_t m = blockIdx.y;
+    const uint64_t blk = blockIdx.x;
+    const uint64_t seg = (a.block + kTile - 1) / kTile;                 // tiles per block, <= 1024
+    const uint64_t t0 = blk * seg;
+    const uint64_t t1 = (t0 + seg < a.ntile) ? t0 + seg : a.ntile;
+    const float* row = a.grads + (uint64_t)m * a.ld;
+    const float mu = (NORM == TNG_NORM_MEAN) ? __ldg(a.means + m) : 0.0f;
+    constexpr int kWords = 4 * CODEC;
+
+    // the lane's four normalised values of tile T, and which of them exist
+    auto tile_values = [&](const uint64_t T, float (&v)[4], uint32_t& valid) {
+        const uint64_t i0 = T * kTile + (uint64_t)lane * 4u;
+        valid = 0;
+#pragma unroll
+        for (int c = 0; c < 4; ++c) valid |= (i0 + c < a.d) ? (1u << c) : 0u;
+        const float4 g = load4(row, i0, a.d);
+        float4 r = make_float4(0.f, 0.f, 0.f, 0.f), r2 = r;
+        if (NORM != TNG_NORM_NONE && NORM != TNG_NORM_MEAN) {
+            if (a.ref) r = load4(a.ref, i0, a.d);
+            if (NORM == TNG_NORM_COMB && a.ref2) r2 = load4(a.ref2, i0, a.d);
+        }
+        NormOp op = make_norm_op<NORM>(r, r2, a.quot_eps);
+        if (NORM == TNG_NORM_MEAN)   // elements past the end read as zero and stay zero
+            op.a = make_float4((valid & 1u) ? mu : 0.0f, (valid & 2u) ? mu : 0.0f, (valid & 4u) ? mu : 0.0f, (valid & 8u) ? mu : 0.0f);
+        encode_normalise<NORM>(g, op, v);
+    };
+
+    for (int i = threadIdx.x; i < 1024; i += 256) buf[i] = 0.0f;
+    __syncthreads();
+    for (uint64_t T = t0 + (uint32_t)warp; T < t1; T += 8) {
+        float v[4];
+        uint32_t valid;
+        tile_values(T, v, valid);
+        const float st = encode_tile_stat<SCALE>(v);
+        if (lane == 0) buf[T - t0] = st;
+    }
+    __syncthreads();
+    cta_tree_1024<SCALE>(buf);
+    const float R = (SCALE == 0) ? buf[0] : __fsqrt_rn(buf[0]);
+    if (threadIdx.x == 0) {
+        a.scales[(uint64_t)m * a.nblk + blk] = R;
+        if (!(fabsf(R) < __int_as_float(0x7f800000))) atomicAdd(a.nonfinite, 1ull);
+    }
+    const float Rq = (SCALE == 1 && !(R > 0.0f)) ? __int_as_float(0x7fc00000) : R;
+    for (uint64_t T = t0 + (uint32_t)warp; T < t1; T += 8) {
+        float v[4];
+        uint32_t valid;
+        tile_values(T, v, valid);
+        const uint64_t q = (T + a.tile0) * 32u + (uint32_t)lane;
+        const uint4 x = philox4x32_10_rk((uint32_t)q, (uint32_t)(q >> 32), a.m_base + m, a.step, a.rk);
+        uint32_t w[kWords];
+        encode_quantise<CODEC, false>(a, v, Rq, x, valid, w);
+        if (lane == 0) {
+            uint4* dst = reinterpret_cast<uint4*>(a.codes + ((uint64_t)m * a.wpw + T * (uint64_t)kWords));
+#pragma unroll
+            for (int q4 = 0; q4 < CODEC; ++q4) dst[q4] = make_uint4(w[4 * q4], w[4 * q4 + 1], w[4 * q4 + 2], w[4 * q4 + 3]);
+        }
+    }
+}
+
+template <int CODEC, int NORM>
+cudaError_t encode_block_cta_scale(const EncodeArgs& a, int scale, dim3 grid, cudaStream_t st) {
+    if (scale == 0) encode_block_cta_kernel<CODEC, NORM, 0><<<grid, 256, 0, st>>>(a);
+    else encode_block_cta_kernel<CODEC, NORM, 1><<<grid, 256, 0, st>>>(a);
+    return cudaGetLastError();
+}
+template <int CODEC>
+cudaError_t encode_block_cta_norm(const EncodeArgs& a, int norm, int scale, dim3 grid, cudaStream_t st) {
+    switch (norm) {
+        case TNG_NORM_DIFF: return encode_block_cta_scale<CODEC, TNG_NORM_DIFF>(a, scale, grid, st);
+        case TNG_NORM_QUOT: return encode_block_cta_scale<CODEC, TNG_NORM_QUOT>(a, scale, grid, st);
+        case TNG_NORM_COMB: return encode_block_cta_scale<CODEC, TNG_NORM_COMB>(a, scale, grid, st);
+        case TNG_NORM_MEAN: return encode_block_cta_scale<CODEC, TNG_NORM_MEAN>(a, scale, grid, st);
+        default: return encode_block_cta_scale<CODEC, TNG_NORM_NONE>(a, scale, grid, st);
+    }
+}
+cudaError_t encode_block_cta_dispatch(const EncodeArgs& a, int codec, int norm, int scale, dim3 grid, cudaStream_t st) {
+    switch (codec) {
+        case TNG_CODEC_SIGN1: return encode_block_cta_norm<TNG_CODEC_SIGN1>(a, norm, scale, grid, st);
+        case TNG_CODEC_TERN2: return encode_block_cta_norm<TNG_CODEC_TERN2>(a, norm, scale, grid, st);
+        default: return encode_block_cta_norm<TNG_CODEC_QSGD4>(a, norm, scale, grid, st);
     }
 }
 
@@ -903,6 +1160,65 @@ cudaError_t encode_launch_tiles(const EncodeArgs& a0, int sm_count, cudaStream_t
     return encode_launch_direct<CODEC, NORM, SCALE, kPhaseFused, FUSEREF>(a, sm_count, st);
 }
 
+// A scale per 256 .. 2048 coordinates: the whole chunks through the staged kernel that shares tile
+// statistics between the warps of a block.  The caller handles the coordinates after the last whole chunk.
+template <int CODEC, int NORM, int SCALE, bool FUSEREF>
+cudaError_t encode_launch_blocks(const EncodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
+    const uint64_t nchunks = a.d / EncGeom::kChunk;
+    static PerDevice<bool> configured;
+    auto kern = encode_pipe_blocks_kernel<CODEC, NORM, SCALE, FUSEREF>;
+    const int slot = device_slot();
+    if (slot < 0 || !configured.v[slot]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)EncGeom::kSmemBytes);
+        if (e != cudaSuccess) return e;
+        if (slot >= 0) configured.v[slot] = true;
+    }
+    EncodePipeArgs pa;
+    pa.e = a;
+    pa.e.tile_begin = nchunks * kEncPipeWarps;
+    pa.rows.nrows = 0;
+    if (FUSEREF) {
+        for (int j = 0; j < a.hist_k; ++j) pa.rows.row[pa.rows.nrows++] = a.hist[j];
+    } else if (NORM != TNG_NORM_NONE && NORM != TNG_NORM_MEAN && a.ref) {
+        pa.rows.row[pa.rows.nrows++] = a.ref;
+        if (NORM == TNG_NORM_COMB && a.ref2) pa.rows.row[pa.rows.nrows++] = a.ref2;
+    }
+    pa.rows.n_pre = pa.rows.nrows;
+    for (uint32_t m = 0; m < a.M; ++m) pa.rows.row[pa.rows.nrows++] = a.grads + (uint64_t)m * a.ld;
+    const int grid = (int)(nchunks < (uint64_t)sm_count ? nchunks : (uint64_t)sm_count);
+    kern<<<grid, kEncPipeThreads, EncGeom::kSmemBytes, st>>>(pa);
+    ++*launches;
+    return cudaGetLastError();
+}
+template <int CODEC, int NORM, int SCALE>
+cudaError_t encode_blocks_fuse(const EncodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
+    if constexpr (NORM != TNG_NORM_NONE && NORM != TNG_NORM_MEAN) {
+        if (a.hist_k > 0) return encode_launch_blocks<CODEC, NORM, SCALE, true>(a, sm_count, st, launches);
+    }
+    return encode_launch_blocks<CODEC, NORM, SCALE, false>(a, sm_count, st, launches);
+}
+template <int CODEC, int NORM>
+cudaError_t encode_blocks_scale(const EncodeArgs& a, int scale, int sm_count, cudaStream_t st, int* launches) {
+    return scale == 0 ? encode_blocks_fuse<CODEC, NORM, 0>(a, sm_count, st, launches) : encode_blocks_fuse<CODEC, NORM, 1>(a, sm_count, st, launches);
+}
+template <int CODEC>
+cudaError_t encode_blocks_norm(const EncodeArgs& a, int norm, int scale, int sm_count, cudaStream_t st, int* launches) {
+    switch (norm) {
+        case TNG_NORM_DIFF: return encode_blocks_scale<CODEC, TNG_NORM_DIFF>(a, scale, sm_count, st, launches);
+        case TNG_NORM_QUOT: return encode_blocks_scale<CODEC, TNG_NORM_QUOT>(a, scale, sm_count, st, launches);
+        case TNG_NORM_COMB: return encode_blocks_scale<CODEC, TNG_NORM_COMB>(a, scale, sm_count, st, launches);
+        case TNG_NORM_MEAN: return encode_blocks_scale<CODEC, TNG_NORM_MEAN>(a, scale, sm_count, st, launches);
+        default: return encode_blocks_scale<CODEC, TNG_NORM_NONE>(a, scale, sm_count, st, launches);
+    }
+}
+cudaError_t encode_blocks_dispatch(const EncodeArgs& a, int codec, int norm, int scale, int sm_count, cudaStream_t st, int* launches) {
+    switch (codec) {
+        case TNG_CODEC_SIGN1: return encode_blocks_norm<TNG_CODEC_SIGN1>(a, norm, scale, sm_count, st, launches);
+        case TNG_CODEC_TERN2: return encode_blocks_norm<TNG_CODEC_TERN2>(a, norm, scale, sm_count, st, launches);
+        default: return encode_blocks_norm<TNG_CODEC_QSGD4>(a, norm, scale, sm_count, st, launches);
+    }
+}
+
 template <int CODEC, int NORM, int SCALE, int PHASE>
 cudaError_t encode_launch(const EncodeArgs& a, int sm_count, cudaStream_t st, int* launches) {
     if constexpr (PHASE == kPhaseFused) {
@@ -986,7 +1302,12 @@ size_t tree_tmp_floats(const CodecGeom& g) {
 
 bool encode_needs_tile_stat(const CodecGeom& g) { return g.block != kTile || g.norm == TNG_NORM_MEAN; }
 
-bool encode_can_fuse_reference(const CodecGeom& g) { return g.block == kTile && g.norm != TNG_NORM_NONE && g.norm != TNG_NORM_MEAN; }
+bool encode_can_fuse_reference(const CodecGeom& g) { return g.norm != TNG_NORM_NONE && g.norm != TNG_NORM_MEAN; }
+
+constexpr uint64_t kShortProblemTiles = 16384;   // tiles x workers up to which the one-launch path is taken
+
+// scale blocks of 2, 4, 8 or 16 tiles lie inside one chunk of the staged pass
+static bool block_within_chunk(uint64_t block) { return block == 256 || block == 512 || block == 1024 || block == 2048; }
 
 cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grads, uint64_t ld, const float* ref, const float* ref2,
                           const RefFusion* fusion,
@@ -1035,20 +1356,60 @@ cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grad
         }
     }
     if (g.block == kTile) return encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseFused, sm_count, st, launches);
-    // general block size: per-tile statistic -> per-block tree -> quantise
+    // A scale per 256 .. 2048 coordinates of a long vector: the whole chunks in one pass over the rows.
+    uint64_t tile_begin = 0;
+    const uint64_t nchunks = g.d / EncGeom::kChunk;
+    if (block_within_chunk(g.block) && nchunks >= kEncPipeMinChunks) {
+        e = encode_blocks_dispatch(a, g.codec, g.norm, g.scale_kind, sm_count, st, launches);
+        if (e != cudaSuccess) return e;
+        tile_begin = nchunks * kEncPipeWarps;
+        if (tile_begin >= g.ntile) return cudaSuccess;
+    }
+    // The remaining coordinates (all of them for any other block size), as a problem of its own that starts at
+    // coordinate i_begin (a multiple of the block): per-tile statistic -> per-block tree -> quantise.
+    const uint64_t i_begin = tile_begin * kTile;
+    if (a.hist_k > 0) {   // the reference was left to this pass: combine what the staged kernel did not
+        const float* rows[kMaxK];
+        for (int j = 0; j < a.hist_k; ++j) rows[j] = a.hist[j] + i_begin;
+        e = launch_combine(rows, a.hist_k, g.d - i_begin, fb, a.ref_out + i_begin, a.ref2_out ? a.ref2_out + i_begin : nullptr,
+                           sm_count, st, launches);
+        if (e != cudaSuccess) return e;
+        a.ref = a.ref_out;
+        if (a.ref2_out) a.ref2 = a.ref2_out;
+        a.hist_k = 0;
+    }
+    const uint64_t blk_begin = i_begin / g.block;
+    const uint64_t nblk_rest = g.nblk - blk_begin;
+    a.grads += i_begin;
+    if (a.ref) a.ref += i_begin;
+    if (a.ref2) a.ref2 += i_begin;
+    a.codes += tile_begin * 4u * (uint64_t)g.codec;
+    a.scales += blk_begin;
+    a.d = g.d - i_begin;
+    a.ntile = g.ntile - tile_begin;       // also the row stride of the tile statistics
+    a.tile0 = g.tile0 + tile_begin;
+    a.tile_begin = 0;
+    // Short problem: one launch, a CTA per (scale block, worker), when a block has at most 1024 tiles and
+    // there are few enough tiles that launch latency, not bandwidth, is what the three-launch path costs.
+    const uint64_t tiles_per_block = (g.block + kTile - 1) / kTile;
+    if (tiles_per_block <= 1024 && a.ntile * (uint64_t)g.M <= kShortProblemTiles && nblk_rest <= 65535) {
+        dim3 grid((unsigned)nblk_rest, g.M);
+        ++*launches;
+        return encode_block_cta_dispatch(a, g.codec, g.norm, g.scale_kind, grid, st);
+    }
     e = encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseStat, sm_count, st, launches);
     if (e != cudaSuccess) return e;
     const float* in = tile_stat;
-    uint64_t n_in = g.ntile;
+    uint64_t n_in = a.ntile;
     uint64_t seg = (g.block + kTile - 1) / kTile;
     float* ping = tree_tmp;
     float* pong = tree_tmp + tree_tmp_floats(g) / 2;
     for (;;) {
         const uint64_t chunks = (seg + 1023) / 1024;
         const int final = chunks == 1;
-        float* out = final ? scales : ping;
-        const uint64_t n_out = g.nblk * chunks;
-        dim3 grid3((unsigned)g.nblk, (unsigned)chunks, g.M);
+        float* out = final ? a.scales : ping;
+        const uint64_t n_out = final ? g.nblk : nblk_rest * chunks;   // row stride: the wire's for the scales themselves
+        dim3 grid3((unsigned)nblk_rest, (unsigned)chunks, g.M);
         if (g.scale_kind == 0)
             block_scale_level_kernel<0><<<grid3, 256, 0, st>>>(in, n_in, seg, chunks, out, n_out, final, 1.0f, &fb->nonfinite);
         else

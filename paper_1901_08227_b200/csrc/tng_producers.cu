@@ -19,12 +19,14 @@ constexpr int kMaxRowChunks = 64;
 template <bool VEC>
 __global__ void __launch_bounds__(256) logistic_margin_kernel(const float* __restrict__ X, const float* __restrict__ b,
                                                               const float* __restrict__ w, uint64_t n, uint64_t d,
-                                                              float* __restrict__ coef, float* __restrict__ lossrow) {
-    __shared__ float part[8];
+                                                              double* __restrict__ coef, float* __restrict__ lossrow) {
+    // The pass is bound by reading the features, so the sums can afford double precision: margins,
+    // sigmoid and the coefficients the transposed product uses are then good to fp32's last place.
+    __shared__ double part[8];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     for (uint64_t i = blockIdx.x; i < n; i += gridDim.x) {
         const float* row = X + i * d;
-        float acc0 = 0.f, acc1 = 0.f, acc2 = 0.f, acc3 = 0.f;
+        double acc0 = 0.0, acc1 = 0.0, acc2 = 0.0, acc3 = 0.0;
         if (VEC) {
             const float4* r4 = reinterpret_cast<const float4*>(row);
             const float4* w4 = reinterpret_cast<const float4*>(w);
@@ -32,33 +34,33 @@ __global__ void __launch_bounds__(256) logistic_margin_kernel(const float* __res
             for (uint64_t j = threadIdx.x; j < d / 4; j += 256) {
                 const float4 x = __ldcs(r4 + j);
                 const float4 ww = __ldg(w4 + j);
-                acc0 = fmaf(x.x, ww.x, acc0); acc1 = fmaf(x.y, ww.y, acc1);
-                acc2 = fmaf(x.z, ww.z, acc2); acc3 = fmaf(x.w, ww.w, acc3);
+                acc0 = fma((double)x.x, (double)ww.x, acc0); acc1 = fma((double)x.y, (double)ww.y, acc1);
+                acc2 = fma((double)x.z, (double)ww.z, acc2); acc3 = fma((double)x.w, (double)ww.w, acc3);
             }
         } else {
-            for (uint64_t j = threadIdx.x; j < d; j += 256) acc0 = fmaf(__ldcs(row + j), __ldg(w + j), acc0);
+            for (uint64_t j = threadIdx.x; j < d; j += 256) acc0 = fma((double)__ldcs(row + j), (double)__ldg(w + j), acc0);
         }
-        float z = (acc0 + acc1) + (acc2 + acc3);
+        double z = (acc0 + acc1) + (acc2 + acc3);
 #pragma unroll
         for (int off = 16; off > 0; off >>= 1) z += __shfl_xor_sync(kFullMask, z, off);
         if (lane == 0) part[warp] = z;
         __syncthreads();
         if (threadIdx.x == 0) {
             z = ((part[0] + part[1]) + (part[2] + part[3])) + ((part[4] + part[5]) + (part[6] + part[7]));
-            const float bi = b[i];
-            const float t = -bi * z;                       // sigma(t), softplus(t), overflow-safe
-            float sig, sp;
-            if (t >= 0.f) {
-                const float e = expf(-t);
-                sig = 1.0f / (1.0f + e);
-                sp = t + log1pf(e);
+            const double bi = (double)b[i];
+            const double t = -bi * z;                      // sigma(t), softplus(t), overflow-safe
+            double sig, sp;
+            if (t >= 0.0) {
+                const double e = exp(-t);
+                sig = 1.0 / (1.0 + e);
+                sp = t + log1p(e);
             } else {
-                const float e = expf(t);
-                sig = e / (1.0f + e);
-                sp = log1pf(e);
+                const double e = exp(t);
+                sig = e / (1.0 + e);
+                sp = log1p(e);
             }
             coef[i] = -bi * sig;
-            lossrow[i] = sp;
+            lossrow[i] = (float)sp;
         }
         __syncthreads();
     }
@@ -66,38 +68,39 @@ __global__ void __launch_bounds__(256) logistic_margin_kernel(const float* __res
 
 // ---- logistic: transposed GEMV, rows split into chunks -----------------------------
 template <bool VEC>
-__global__ void __launch_bounds__(256) logistic_colsum_kernel(const float* __restrict__ X, const float* __restrict__ coef,
+__global__ void __launch_bounds__(256) logistic_colsum_kernel(const float* __restrict__ X, const double* __restrict__ coef,
                                                               uint64_t n, uint64_t d, uint64_t rows_per_chunk,
-                                                              float* __restrict__ partial) {
+                                                              double* __restrict__ partial) {
     const uint64_t col = ((uint64_t)blockIdx.x * blockDim.x + threadIdx.x) * (VEC ? 4 : 1);
     if (col >= d) return;
     const uint64_t r0 = (uint64_t)blockIdx.y * rows_per_chunk;
     const uint64_t r1 = (r0 + rows_per_chunk < n) ? r0 + rows_per_chunk : n;
     if (VEC) {
-        float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+        double a0 = 0.0, a1 = 0.0, a2 = 0.0, a3 = 0.0;
 #pragma unroll 8
         for (uint64_t i = r0; i < r1; ++i) {
-            const float ci = __ldg(coef + i);
+            const double ci = __ldg(coef + i);
             const float4 x = __ldcs(reinterpret_cast<const float4*>(X + i * d + col));
-            acc.x = fmaf(ci, x.x, acc.x); acc.y = fmaf(ci, x.y, acc.y);
-            acc.z = fmaf(ci, x.z, acc.z); acc.w = fmaf(ci, x.w, acc.w);
+            a0 = fma(ci, (double)x.x, a0); a1 = fma(ci, (double)x.y, a1);
+            a2 = fma(ci, (double)x.z, a2); a3 = fma(ci, (double)x.w, a3);
         }
-        *reinterpret_cast<float4*>(partial + (uint64_t)blockIdx.y * d + col) = acc;
+        double* dst = partial + (uint64_t)blockIdx.y * d + col;
+        dst[0] = a0; dst[1] = a1; dst[2] = a2; dst[3] = a3;
     } else {
-        float acc = 0.f;
-        for (uint64_t i = r0; i < r1; ++i) acc = fmaf(__ldg(coef + i), __ldcs(X + i * d + col), acc);
+        double acc = 0.0;
+        for (uint64_t i = r0; i < r1; ++i) acc = fma(__ldg(coef + i), (double)__ldcs(X + i * d + col), acc);
         partial[(uint64_t)blockIdx.y * d + col] = acc;
     }
 }
 
-__global__ void __launch_bounds__(256) logistic_finish_kernel(const float* __restrict__ partial, int chunks, uint64_t n,
+__global__ void __launch_bounds__(256) logistic_finish_kernel(const double* __restrict__ partial, int chunks, uint64_t n,
                                                               uint64_t d, const float* __restrict__ w, float lambda2,
                                                               float* __restrict__ grad) {
     const uint64_t j = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     if (j >= d) return;
-    float acc = 0.f;
+    double acc = 0.0;
     for (int c = 0; c < chunks; ++c) acc += partial[(uint64_t)c * d + j];
-    grad[j] = fmaf(lambda2, w[j], acc / (float)n);
+    grad[j] = (float)(acc / (double)n + (double)lambda2 * (double)w[j]);
 }
 
 // single CTA: loss = mean(lossrow) + lambda2/2 ||w||^2, accumulated in double
@@ -207,7 +210,7 @@ bool vec_ok(const float* X, const float* w, uint64_t d) {
     return d % 4 == 0 && (reinterpret_cast<uintptr_t>(X) & 15u) == 0 && (reinterpret_cast<uintptr_t>(w) & 15u) == 0;
 }
 
-cudaError_t launch_margins(const float* X, const float* b, const float* w, uint64_t n, uint64_t d, float* coef,
+cudaError_t launch_margins(const float* X, const float* b, const float* w, uint64_t n, uint64_t d, double* coef,
                            float* lossrow, cudaStream_t st) {
     const uint64_t cap = (uint64_t)sm_count_now() * 64u;
     const int grid = (int)(n < cap ? n : cap);
@@ -223,10 +226,10 @@ using namespace tng;
 
 extern "C" {
 
+// scratch layout (in floats): coef as n4 doubles, lossrow as n4 floats, partial as kMaxRowChunks x d doubles
 size_t tng_logistic_scratch_floats(uint64_t n, uint64_t d) {
-    // coef[n], lossrow[n] (rounded up to a multiple of 4 each), partial[kMaxRowChunks][d]
     const uint64_t n4 = (n + 3) / 4 * 4;
-    return (size_t)(2 * n4 + (uint64_t)kMaxRowChunks * d);
+    return (size_t)(3 * n4 + 2 * (uint64_t)kMaxRowChunks * d);
 }
 
 tng_status tng_logistic_grad(const float* X_dev, const float* b_dev, uint64_t n, uint64_t d, const float* w_dev,
@@ -235,9 +238,9 @@ tng_status tng_logistic_grad(const float* X_dev, const float* b_dev, uint64_t n,
     if ((reinterpret_cast<uintptr_t>(scratch_dev) & 15u) != 0) return TNG_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint64_t n4 = (n + 3) / 4 * 4;
-    float* coef = scratch_dev;
-    float* lossrow = scratch_dev + n4;
-    float* partial = scratch_dev + 2 * n4;
+    double* coef = reinterpret_cast<double*>(scratch_dev);
+    float* lossrow = scratch_dev + 2 * n4;
+    double* partial = reinterpret_cast<double*>(scratch_dev + 3 * n4);   // n4 is a multiple of 4: 16-byte aligned
     if (launch_margins(X_dev, b_dev, w_dev, n, d, coef, lossrow, st) != cudaSuccess) return TNG_ERR_CUDA;
     const bool vec = vec_ok(X_dev, w_dev, d);
     const int chunks = row_chunks(n, d, vec);
@@ -256,8 +259,8 @@ tng_status tng_logistic_loss(const float* X_dev, const float* b_dev, uint64_t n,
     if ((reinterpret_cast<uintptr_t>(scratch_dev) & 15u) != 0) return TNG_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     const uint64_t n4 = (n + 3) / 4 * 4;
-    float* coef = scratch_dev;
-    float* lossrow = scratch_dev + n4;
+    double* coef = reinterpret_cast<double*>(scratch_dev);
+    float* lossrow = scratch_dev + 2 * n4;
     if (launch_margins(X_dev, b_dev, w_dev, n, d, coef, lossrow, st) != cudaSuccess) return TNG_ERR_CUDA;
     logistic_loss_kernel<<<1, 1024, 0, st>>>(lossrow, n, w_dev, d, lambda2, loss_dev);
     return cudaGetLastError() == cudaSuccess ? TNG_OK : TNG_ERR_CUDA;

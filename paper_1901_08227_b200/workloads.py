@@ -117,10 +117,14 @@ class GradientStream:
         self.mu = self.rho * self.mu + math.sqrt(1.0 - self.rho ** 2) * self.scale * eps
         return self.mu
 
-    def worker_grads(self, out=None):
+    def worker_grads(self, out=None, first=0, count=None):
+        """Rows of workers first .. first + count - 1 (default: all M).  A worker's row depends on
+        (seed, step, worker) only, so ranks that hold different workers draw consistent rows."""
+        count = self.M - first if count is None else count
         if out is None:
-            out = torch.empty((self.M, self.d), dtype=torch.float32, device=self.device)
-        for m in range(self.M):
+            out = torch.empty((count, self.d), dtype=torch.float32, device=self.device)
+        for r in range(count):
+            m = first + r
             stream = 100000 + self.t * 128 + m
             z = normal((self.d,), self.seed, stream, self.device)
             chi = torch.zeros_like(z)
@@ -129,7 +133,7 @@ class GradientStream:
                 chi.addcmul_(w, w)
             chi.div_(float(self.nu)).sqrt_()
             z.div_(chi).mul_(self.scale).add_(self.mu)
-            out[m].copy_(z)
+            out[r].copy_(z)
         return out
 
 

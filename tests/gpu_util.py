@@ -31,7 +31,16 @@ def same_bits(a, b):
 
 
 def same_values(a, b):
-    """equal as numbers, NaN == NaN"""
+    """float arrays equal bit for bit (+0 and -0 differ), except that a NaN equals a NaN whatever its payload"""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    b = np.ascontiguousarray(b, dtype=np.float32)
+    if a.shape != b.shape:
+        return False
+    return bool(np.all((a.view(np.uint32) == b.view(np.uint32)) | (np.isnan(a) & np.isnan(b))))
+
+
+def same_numbers(a, b):
+    """equal as numbers (+0 == -0), NaN == NaN"""
     return np.array_equal(np.asarray(a), np.asarray(b), equal_nan=True)
 
 

@@ -65,6 +65,20 @@ def test_general_block_sizes_bit_exact(codec, scale_kind, B, d):
 
 
 @pytest.mark.parametrize("codec", CODECS)
+@pytest.mark.parametrize("scale_kind", [0, 1])
+@pytest.mark.parametrize("B,d,M,norm", [(256, 2048 * 9 + 50, 8, tng.NORM_DIFF), (512, 2048 * 8, 3, tng.NORM_QUOT),
+                                        (1024, 2048 * 11 + 1024 + 384 + 7, 13, tng.NORM_DIFF), (2048, 2048 * 10 + 2047, 5, tng.NORM_NONE),
+                                        (256, 2048 * 12 + 128, 64, tng.NORM_QUOT), (2048, 2048 * 150 + 300, 2, tng.NORM_DIFF)])
+def test_blocks_of_several_tiles_in_long_vectors_take_one_pass(codec, scale_kind, B, d, M, norm):
+    # a scale per 256 .. 2048 coordinates of a vector of at least 8 chunks: the whole chunks go through the
+    # staged kernel whose warps share tile statistics, the rest (whole blocks and a ragged one) through
+    # the three-launch path; neither wire nor aggregate may show the seam
+    got, want, st = run_both(d, M, codec, norm, B, scale_kind=scale_kind, s=6)
+    assert st.pipeline_error == 0
+    assert_exact(got, want)
+
+
+@pytest.mark.parametrize("codec", CODECS)
 @pytest.mark.parametrize("norm", [tng.NORM_DIFF, tng.NORM_QUOT])
 def test_l2_scale_block128(codec, norm):
     got, want, _ = run_both(5000, 4, codec, norm, 128, scale_kind=1)

@@ -1,6 +1,6 @@
 """GPU parity at the benchmark's full size and launch configuration: d = 2^27 coordinates,
 M = 8 workers, K = 8 ring entries, quotient form, ternary codes, one scale per 128
-coordinates, least-squares fusion -- one whole round through tng_step, as bench.py times it.
+coordinates, least-squares fusion -- whole rounds through tng_step, as bench.py times them.
 
 The fusion statistics are global sums, so the oracle computes them on the whole vectors; the
 reference, the wire and the aggregate are checked bit for bit on sampled windows of
@@ -19,29 +19,12 @@ pytestmark = pytest.mark.gpu
 D, M, K = 1 << 27, 8, 8
 
 
-def test_full_size_round_in_the_benchmark_configuration():
-    free, _ = torch.cuda.mem_get_info()
-    if free < 24 * (1 << 30):
-        pytest.skip("needs about 24 GiB of free device memory")
-    dev = "cuda"
-    stream = workloads.GradientStream(0, D, M, device=dev)
-    ctx = tng.Context(D, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, block=128, fuse_mode=tng.FUSE_LSQ)
-    hist = []                                         # host copies, oldest first
-    for _ in range(K):
-        mu = stream.advance()
-        ctx.push_reference(mu)
-        hist.append(to_np(mu))
-    hist = hist[::-1]                                 # newest first, as the fusion numbers them
-    stream.advance()
-    g = stream.worker_grads()
-    del stream
-    out = torch.empty(D, device=dev)
-    ctx.step(g, out)
-    torch.cuda.synchronize()
+def check_round(ctx, hist, g, out, step, rng):
+    """One finished round against the oracle: `hist` are host copies of the ring as it stood before the
+    round (newest first), `g` the round's gradient rows, `out` its aggregate, `step` its round number."""
     st = ctx.stats()
     assert st.pipeline_error == 0 and st.solver_fallback == 0 and st.nonfinite_scales == 0
-    assert st.rounds == 1 and st.k == K
-
+    assert st.rounds == step + 1 and st.k == K
     # ---- fusion statistics and coefficients against the oracle on the whole vectors
     gn = to_np(g)
     oG, oc, ogg = oracle.fuse_stats(hist, gn)
@@ -59,7 +42,6 @@ def test_full_size_round_in_the_benchmark_configuration():
     ref = ctx.reference()
     codes, scales = ctx.wire()
     newest = ctx.history(0)
-    rng = np.random.default_rng(0)
     windows = [(0, 2048), (D - 2048, 2048), (2048 * 148 - 256, 512), (2048 * 149 * 7 - 128, 256)]
     windows += [(int(t) * 128, 1024) for t in rng.integers(0, D // 128 - 8, size=60)]
     for i0, n in windows:
@@ -68,7 +50,7 @@ def test_full_size_round_in_the_benchmark_configuration():
         got_ref = to_np(ref[sl])
         assert np.array_equal(got_ref.view(np.uint32), want_ref.view(np.uint32)), f"reference differs in window {i0}"
         wc, ws = oracle.encode(np.ascontiguousarray(gn[:, sl]), want_ref, tng.NORM_QUOT, tng.CODEC_TERN2, B=128, seed=(0, 0),
-                               t=0, coord_offset=i0)
+                               t=step, coord_offset=i0)
         t0, t1 = i0 // 128, (i0 + n) // 128
         assert np.array_equal(to_np(codes[:, t0 * 8:t1 * 8]).view(np.uint32), wc), f"codes differ in window {i0}"
         assert np.array_equal(to_np(scales[:, t0:t1]).view(np.uint32), ws.view(np.uint32)), f"scales differ in window {i0}"
@@ -78,6 +60,37 @@ def test_full_size_round_in_the_benchmark_configuration():
     # ---- properties that hold at any size
     assert bool(torch.isfinite(out).all())
     assert bool((scales >= 0).all())
+
+
+def test_full_size_rounds_in_the_benchmark_configuration():
+    """K + 2 rounds.  The first one works on a ring seeded with the stream's means; by the last one every
+    ring entry is an aggregate the library decoded itself.  Both are checked against the oracle."""
+    free, _ = torch.cuda.mem_get_info()
+    if free < 28 * (1 << 30):
+        pytest.skip("needs about 28 GiB of free device memory")
+    dev = "cuda"
+    stream = workloads.GradientStream(0, D, M, device=dev)
+    ctx = tng.Context(D, M, K, tng.CODEC_TERN2, tng.NORM_QUOT, block=128, fuse_mode=tng.FUSE_LSQ)
+    hist = []                                         # host copies, oldest first
+    for _ in range(K):
+        mu = stream.advance()
+        ctx.push_reference(mu)
+        hist.append(to_np(mu))
+    hist = hist[::-1]                                 # newest first, as the fusion numbers them
+    out = torch.empty(D, device=dev)
+    rng = np.random.default_rng(0)
+    rounds = K + 2
+    for step in range(rounds):
+        stream.advance()
+        g = stream.worker_grads()
+        if step == rounds - 1:                        # the ring as it stands: the library's own aggregates
+            torch.cuda.synchronize()
+            hist = [to_np(ctx.history(j)) for j in range(K)]
+        ctx.step(g, out)
+        torch.cuda.synchronize()
+        if step == 0 or step == rounds - 1:
+            check_round(ctx, hist, g, out, step, rng)
+        del g
     ctx.close()
 
 

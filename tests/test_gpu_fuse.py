@@ -5,7 +5,7 @@ import pytest
 import torch
 
 import oracle
-from gpu_util import codes_np, drifting_grads, make_ctx, make_oracle, rel_l2, same_values, to_np
+from gpu_util import same_numbers, codes_np, drifting_grads, make_ctx, make_oracle, rel_l2, same_values, to_np
 from paper_1901_08227_b200 import tng, workloads
 
 pytestmark = pytest.mark.gpu
@@ -94,7 +94,12 @@ def test_rounds_are_bit_exact_when_the_reference_is(mode, K, norm, codec, B, d):
         if not (mode == tng.FUSE_LAST and K == 1):
             # (with K = 1 the delayed-gradient reference aliases the only ring slot, which the
             # round has just overwritten with the new aggregate)
-            assert same_values(to_np(ctx.reference()), orc.ref())
+            # The delayed-gradient reference IS the newest ring entry on the GPU (no pass), while the oracle
+            # forms fma(1, h, +0): a -0 entry stays -0 on one side and becomes +0 on the other.  Nothing the
+            # round computes depends on the sign of a zero reference element (the aggregates above are
+            # compared bit for bit), so the reference itself is compared as numbers there.
+            same = same_numbers if mode == tng.FUSE_LAST else same_values
+            assert same(to_np(ctx.reference()), orc.ref())
     st = ctx.stats()
     assert st.rounds == steps and st.k == min(steps, K) and st.kernel_launches > 0
 

@@ -4,7 +4,7 @@ import numpy as np
 import pytest
 import torch
 
-from gpu_util import codes_np, drifting_grads, make_ctx, make_oracle, same_values, to_np
+from gpu_util import codes_np, drifting_grads, make_ctx, make_oracle, same_numbers, same_values, to_np
 from paper_1901_08227_b200 import tng
 
 pytestmark = pytest.mark.gpu
@@ -24,7 +24,10 @@ def test_refresh_cadence_matches_the_oracle_bit_for_bit(mode, K, norm, codec, B,
         ctx.step(g, out)
         want = orc.step(to_np(g))
         codes, scales = ctx.wire()
-        assert same_values(to_np(ctx.reference()), orc.ref()), f"reference differs at round {t}"
+        # (the delayed-gradient reference is a copy of a ring entry on the GPU and fma(1, h, +0) in the oracle:
+        # they differ in the sign of zeros only, which no result depends on)
+        same = same_numbers if mode == tng.FUSE_LAST else same_values
+        assert same(to_np(ctx.reference()), orc.ref()), f"reference differs at round {t}"
         assert np.array_equal(codes_np(codes), orc.codes()), f"codes differ at round {t}"
         assert same_values(to_np(scales), orc.scales())
         assert same_values(to_np(out), want)

@@ -64,6 +64,34 @@ def test_reference_arm_runs_on_rank_zero_only():
     assert p.returncode == 0 and p.stdout.strip() == ""
 
 
+def test_gpus_flag_starts_its_own_ranks():
+    # `bench.py --gpus 2` without a launcher around it starts two ranks itself (what torchrun would do); the
+    # --rank-check mode runs that path on CPU: the ranks meet over gloo, agree on the slowest rank's time and
+    # assemble a wire block by block, and rank 0 alone prints the line
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    p = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--rank-check"], env=env, capture_output=True,
+                       text=True, timeout=300)
+    assert p.returncode == 0, p.stderr[-2000:]
+    lines = [ln for ln in p.stdout.splitlines() if ln.startswith("{")]
+    assert len(lines) == 1
+    line = json.loads(lines[0])
+    assert line["n_gpus"] == 2 and line["job_ms"] == 2.0 and line["wire_rows"] == [1, 2]
+    # under a launcher (WORLD_SIZE set) the script must not start ranks of its own
+    cmd = bench.launch_command(2, ["--gpus", "2"], 29999)
+    assert cmd[1:4] == ["-m", "torch.distributed.run", "--nnodes=1"] and "--nproc-per-node=2" in cmd and cmd[-2:] == ["--gpus", "2"]
+    assert "127.0.0.1" in cmd
+
+
+def test_exchange_bytes_of_the_splits():
+    # worker split at the headline shape on 8 ranks: each rank sends its worker's codes and scales, 2^27 * 2 / 8 + 2^20 * 4 bytes
+    wpw, nblk = (1 << 27) // 128 * 8, (1 << 27) // 128
+    ex = bench.exchange_bytes("workers", 8, 8, wpw, nblk)
+    assert ex["allreduce_bytes"] == 136 and ex["allgather_send_bytes_per_rank"] == (1 << 25) + (1 << 22)
+    assert ex["allgather_total_bytes"] == 8 * ex["allgather_send_bytes_per_rank"]
+    assert bench.exchange_bytes("coords", 4, 8, wpw, nblk) == {"allreduce_bytes": 2184}
+    assert bench.exchange_bytes("none", 4, 8, wpw, nblk) == {}
+
+
 def test_algorithmic_bytes_of_the_round():
     per = bench.algorithmic_bytes_per_coord(8, 8, 2, 128, "lsq")
     assert per["dots"] == 64.0 and per["encode"] == 70.25 and per["decode"] == 14.25
@@ -76,6 +104,11 @@ def test_algorithmic_bytes_of_the_round():
     assert set(scalar) == {"encode", "decode"} and scalar["encode"] == 66.25 and scalar["decode"] == 10.25
     last = bench.algorithmic_bytes_per_coord(8, 8, 2, 128, "last")                 # the reference is a ring slot: no combine
     assert "dots" not in last and last["encode"] == 38.25
+    # a scale per 256 coordinates is still one read of the rows; one scale per vector needs two
+    b256 = bench.algorithmic_bytes_per_coord(16, 4, 4, 256, "lsq", norm="diff")
+    assert b256["encode"] == 16 + 64 + 4 + 8 + 0.25
+    vec = bench.algorithmic_bytes_per_coord(4, 1, 2, 0, "last", norm="diff")
+    assert vec["encode"] == 2 * (16 + 4) + 1.0 and vec["decode"] == 1.0 + 4 + 4 + 4
 
 
 def _gather_main(rank, world, port, out_dir):
