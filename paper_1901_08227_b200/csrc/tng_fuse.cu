@@ -40,36 +40,36 @@ struct DotsShape {
 
 // CTA reduction (lanes by butterfly, warps in warp order), one partial row per CTA, and
 // the CTA that arrives last adds the partial rows in CTA order: run-to-run identical sums,
-// nobody waits.  `tid` in [0, nthreads) indexes the threads that hold accumulators; every
-// thread of the CTA must call this (it contains __syncthreads), the others with tid >= nthreads.
+// nobody waits.  Called by the kDotsThreads threads that hold accumulators (tid in [0, kDotsThreads)) and
+// by nobody else: its barriers count exactly those threads.
+__device__ __forceinline__ void dots_threads_barrier() {
+    asm volatile("bar.sync 2, %0;" ::"n"(kDotsThreads) : "memory");
+}
 template <int kAcc, int kPairs, bool SAME>
-__device__ __forceinline__ void dots_finish(const double (&acc)[kAcc], const DotsArgs& a, const bool with_g, const int tid,
-                                            const int nthreads) {
+__device__ __forceinline__ void dots_finish(const double (&acc)[kAcc], const DotsArgs& a, const bool with_g, const int tid) {
     __shared__ double warp_part[kDotsThreads / 32][kAcc];
     __shared__ bool is_last;
     const int lane = tid & 31, warp = tid >> 5;
-    if (tid < nthreads) {
 #pragma unroll
-        for (int i = 0; i < kAcc; ++i) {
-            double v = acc[i];
+    for (int i = 0; i < kAcc; ++i) {
+        double v = acc[i];
 #pragma unroll
-            for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(kFullMask, v, off);
-            if (lane == 0) warp_part[warp][i] = v;
-        }
+        for (int off = 16; off > 0; off >>= 1) v += __shfl_xor_sync(kFullMask, v, off);
+        if (lane == 0) warp_part[warp][i] = v;
     }
-    __syncthreads();
+    dots_threads_barrier();
     if (tid < kAcc) {
         double v = 0.0;
-        for (int w = 0; w < nthreads / 32; ++w) v += warp_part[w][tid];
+        for (int w = 0; w < kDotsThreads / 32; ++w) v += warp_part[w][tid];
         a.partials[(uint64_t)blockIdx.x * kDotsMaxAcc + tid] = v;
     }
     __threadfence();
-    __syncthreads();
+    dots_threads_barrier();
     if (tid == 0) {
         const uint32_t prev = atomicAdd(&a.fb->dots_arrivals, 1u);
         is_last = (prev == gridDim.x - 1);
     }
-    __syncthreads();
+    dots_threads_barrier();
     if (!is_last) return;
     __threadfence();
     if (tid < kAcc) {
@@ -89,7 +89,15 @@ __device__ __forceinline__ void dots_finish(const double (&acc)[kAcc], const Dot
 // following fills, and accumulates exactly what dots_kernel accumulates.  The ragged end
 // of the vectors (d mod 1024) is read directly.
 // ---------------------------------------------------------------------------
-constexpr int kDotsPipeThreads = kDotsThreads + 32;   // 8 consumer warps + 1 producer warp
+// 8 consumer warps (two warpgroups) + one warpgroup of which one thread feeds the pipeline.  The kernel starts
+// with kDotsLaunchRegs registers per thread; the feeding warpgroup gives all but kDotsFeedRegs of its share back and
+// the consumers take it (setmaxnreg), so that the 45 double accumulators of eight history rows, the rows' values
+// and the gradient sums fit in registers.  The shares add up exactly:
+//   256 x kDotsConsumerRegs + 128 x kDotsFeedRegs = 384 x kDotsLaunchRegs = 64512  (and, per SM partition, which holds
+//   two consumer warps and one feeding warp: 32 x (2 x 240 + 24) = 16128 <= 16384).
+constexpr int kDotsPipeThreads = kDotsThreads + 128;
+constexpr int kDotsLaunchRegs = 168, kDotsConsumerRegs = 240, kDotsFeedRegs = 24;
+static_assert(kDotsThreads * kDotsConsumerRegs + 128 * kDotsFeedRegs == kDotsPipeThreads * kDotsLaunchRegs, "register shares must add up to what the launch holds");
 using DotsGeom = PipeGeom<1024, 16, 3>;                // 64 KiB stages: a chunk of 1024 coordinates of 16 rows
 constexpr uint64_t kDotsPipeMinCoords = 16 * DotsGeom::kChunk;   // shorter vectors take the direct kernel
 
@@ -98,11 +106,30 @@ struct DotsPipeArgs {
     PipeRows rows;      // history rows then gradient rows
 };
 
+// The sum of the M gradients at a coordinate enters the right-hand side, which decides the coefficients down
+// to their last fp32 bit: it is kept in double, like everything else the coefficients depend on.  The sum
+// of squares only feeds the C_nz estimate: fp32.
+struct GradSums {
+    double sum[4];
+    float4 sq;
+};
+__device__ __forceinline__ void grad_sums(GradSums& a, const float4 g) {
+    a.sum[0] += (double)g.x; a.sum[1] += (double)g.y; a.sum[2] += (double)g.z; a.sum[3] += (double)g.w;
+    a.sq.x = fmaf(g.x, g.x, a.sq.x); a.sq.y = fmaf(g.y, g.y, a.sq.y); a.sq.z = fmaf(g.z, g.z, a.sq.z); a.sq.w = fmaf(g.w, g.w, a.sq.w);
+}
+__device__ __forceinline__ GradSums grad_sums_zero() {
+    GradSums a;
+    a.sum[0] = a.sum[1] = a.sum[2] = a.sum[3] = 0.0;
+    a.sq = make_float4(0.f, 0.f, 0.f, 0.f);
+    return a;
+}
+
 // acc += products of the four coordinates held in ha[] (history) and gs/gq (sum and sum of
 // squares of the gradients at these coordinates, fp32, m ascending)
 template <int NA>
-__device__ __forceinline__ void dots_accum4(const float4 (&ha)[NA], const float4 gs, const float4 gq, const bool with_g,
+__device__ __forceinline__ void dots_accum4(const float4 (&ha)[NA], const GradSums& gsum, const bool with_g,
                                             double (&acc)[NA * (NA + 1) / 2 + NA + 1]) {
+    const float4 gq = gsum.sq;
     constexpr int kPairs = NA * (NA + 1) / 2;
 #pragma unroll
     for (int comp = 0; comp < 4; ++comp) {
@@ -115,7 +142,7 @@ __device__ __forceinline__ void dots_accum4(const float4 (&ha)[NA], const float4
 #pragma unroll
             for (int j = i; j < NA; ++j) { acc[p] = fma(da[i], da[j], acc[p]); ++p; }
         if (with_g) {
-            const double dg = (double)(comp == 0 ? gs.x : comp == 1 ? gs.y : comp == 2 ? gs.z : gs.w);
+            const double dg = gsum.sum[comp];
 #pragma unroll
             for (int i = 0; i < NA; ++i) acc[kPairs + i] = fma(da[i], dg, acc[kPairs + i]);
             acc[kPairs + NA] += (double)(comp == 0 ? gq.x : comp == 1 ? gq.y : comp == 2 ? gq.z : gq.w);
@@ -123,10 +150,6 @@ __device__ __forceinline__ void dots_accum4(const float4 (&ha)[NA], const float4
     }
 }
 
-__device__ __forceinline__ void grad_sums(float4& gs, float4& gq, const float4 g) {
-    gs.x += g.x; gs.y += g.y; gs.z += g.z; gs.w += g.w;
-    gq.x = fmaf(g.x, g.x, gq.x); gq.y = fmaf(g.y, g.y, gq.y); gq.z = fmaf(g.z, g.z, gq.z); gq.w = fmaf(g.w, g.w, gq.w);
-}
 
 template <int NA>
 __global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const DotsPipeArgs pa) {
@@ -139,17 +162,20 @@ __global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const Do
     const bool with_g = a.grads != nullptr;
     const uint64_t nchunks = a.d / G::kChunk;
     const int tid = threadIdx.x;
-    double acc[kAcc];
-#pragma unroll
-    for (int i = 0; i < kAcc; ++i) acc[i] = 0.0;
-
     if (tid >= kDotsThreads) {
-        // ---- producer warp: one thread feeds the stages
+        // ---- the feeding warpgroup: hands its registers over, then one thread feeds the stages
+        asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kDotsFeedRegs));
         if (tid == kDotsThreads) {
             const uint32_t err = pipe_produce<G>(pipe, pa.rows, blockIdx.x, gridDim.x, nchunks);
             if (err != kPipeOk) atomicMax(&a.fb->pipe_error, err);
         }
-    } else {
+        return;
+    }
+    asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kDotsConsumerRegs));
+    double acc[kAcc];
+#pragma unroll
+    for (int i = 0; i < kAcc; ++i) acc[i] = 0.0;
+    {
         // ---- consumers: fill 0 of a chunk holds the NA history rows, the others gradient rows
         const int lane = tid & 31;
         const uint32_t my = (uint32_t)tid * 16u;                  // byte offset of the thread's float4 inside a row chunk
@@ -158,7 +184,7 @@ __global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const Do
         bool alive = true;
         for (uint64_t c = blockIdx.x; c < nchunks && alive; c += gridDim.x) {
             float4 ha[NA];
-            float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), gq = make_float4(0.f, 0.f, 0.f, 0.f);
+            GradSums gsum = grad_sums_zero();
             for (int g0 = -G::kRows; g0 < ngrad; g0 += G::kRows) {   // g0 < 0: the history fill
                 const uint32_t s = it % G::kStages, use = it / G::kStages;
                 if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {   // warp-uniform outcome
@@ -172,13 +198,13 @@ __global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const Do
                     for (int j = 0; j < NA; ++j) ha[j] = lds128(base + (uint32_t)j * G::kRowBytes);
                 } else {
                     const int n = (ngrad - g0 < G::kRows) ? ngrad - g0 : G::kRows;
-                    for (int r = 0; r < n; ++r) grad_sums(gs, gq, lds128(base + (uint32_t)r * G::kRowBytes));
+                    for (int r = 0; r < n; ++r) grad_sums(gsum, lds128(base + (uint32_t)r * G::kRowBytes));
                 }
                 __syncwarp();
                 if (lane == 0) mbar_arrive(pipe.empty(s));       // this warp has read the stage
                 ++it;
             }
-            if (alive) dots_accum4<NA>(ha, gs, gq, with_g, acc);
+            if (alive) dots_accum4<NA>(ha, gsum, with_g, acc);
         }
         // ---- ragged end: coordinates [nchunks*1024, d) straight from global memory
         const uint64_t ngroups = (a.d + 3) / 4;
@@ -188,13 +214,13 @@ __global__ void __launch_bounds__(kDotsPipeThreads, 1) dots_pipe_kernel(const Do
             float4 ha[NA];
 #pragma unroll
             for (int j = 0; j < NA; ++j) ha[j] = load4_stream(a.rows_a[j], i0, a.d);
-            float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), gq = make_float4(0.f, 0.f, 0.f, 0.f);
+            GradSums gsum = grad_sums_zero();
             if (with_g)
-                for (uint32_t m = 0; m < a.M; ++m) grad_sums(gs, gq, load4_stream(a.grads + (uint64_t)m * a.ld, i0, a.d));
-            dots_accum4<NA>(ha, gs, gq, with_g, acc);
+                for (uint32_t m = 0; m < a.M; ++m) grad_sums(gsum, load4_stream(a.grads + (uint64_t)m * a.ld, i0, a.d));
+            dots_accum4<NA>(ha, gsum, with_g, acc);
         }
     }
-    dots_finish<kAcc, kPairs, true>(acc, a, with_g, tid, kDotsThreads);
+    dots_finish<kAcc, kPairs, true>(acc, a, with_g, tid);
 }
 
 template <int NA, int NB, bool SAME>
@@ -218,8 +244,8 @@ __global__ void __launch_bounds__(kDotsThreads, 1) dots_kernel(const DotsArgs a)
 #pragma unroll
             for (int j = 0; j < NB; ++j) hb[j] = load4_stream(a.rows_b[j], i0, a.d);
         }
-        // sum and sum of squares of the M gradients at these coordinates (fp32, m ascending)
-        float4 gs = make_float4(0.f, 0.f, 0.f, 0.f), gq = make_float4(0.f, 0.f, 0.f, 0.f);
+        // sum (double) and sum of squares (fp32) of the M gradients at these coordinates, m ascending
+        GradSums gsum = grad_sums_zero();
         if (with_g) {
             for (uint32_t m0 = 0; m0 < a.M; m0 += 8) {
                 float4 g[8];
@@ -228,11 +254,7 @@ __global__ void __launch_bounds__(kDotsThreads, 1) dots_kernel(const DotsArgs a)
                     if (m0 + k < a.M) g[k] = load4_stream(a.grads + (uint64_t)(m0 + k) * a.ld, i0, a.d);
 #pragma unroll
                 for (int k = 0; k < 8; ++k)
-                    if (m0 + k < a.M) {
-                        gs.x += g[k].x; gs.y += g[k].y; gs.z += g[k].z; gs.w += g[k].w;
-                        gq.x = fmaf(g[k].x, g[k].x, gq.x); gq.y = fmaf(g[k].y, g[k].y, gq.y);
-                        gq.z = fmaf(g[k].z, g[k].z, gq.z); gq.w = fmaf(g[k].w, g[k].w, gq.w);
-                    }
+                    if (m0 + k < a.M) grad_sums(gsum, g[k]);
             }
         }
 #pragma unroll
@@ -247,10 +269,10 @@ __global__ void __launch_bounds__(kDotsThreads, 1) dots_kernel(const DotsArgs a)
 #pragma unroll
                     for (int j = i; j < NA; ++j) { acc[p] = fma(da[i], da[j], acc[p]); ++p; }
                 if (with_g) {
-                    const double dg = (double)(comp == 0 ? gs.x : comp == 1 ? gs.y : comp == 2 ? gs.z : gs.w);
+                    const double dg = gsum.sum[comp];
 #pragma unroll
                     for (int i = 0; i < NA; ++i) acc[Shape::kPairs + i] = fma(da[i], dg, acc[Shape::kPairs + i]);
-                    acc[Shape::kPairs + NA] += (double)(comp == 0 ? gq.x : comp == 1 ? gq.y : comp == 2 ? gq.z : gq.w);
+                    acc[Shape::kPairs + NA] += (double)(comp == 0 ? gsum.sq.x : comp == 1 ? gsum.sq.y : comp == 2 ? gsum.sq.z : gsum.sq.w);
                 }
             } else {
                 double db[SAME ? 1 : NB];
@@ -264,7 +286,7 @@ __global__ void __launch_bounds__(kDotsThreads, 1) dots_kernel(const DotsArgs a)
         }
     }
 
-    dots_finish<kAcc, Shape::kPairs, SAME>(acc, a, with_g, threadIdx.x, kDotsThreads);
+    dots_finish<kAcc, Shape::kPairs, SAME>(acc, a, with_g, threadIdx.x);
 }
 
 template <int NA>
@@ -287,6 +309,18 @@ cudaError_t dots_pipe(const DotsPipeArgs& pa, int grid, cudaStream_t st) {
         if (e != cudaSuccess) return e;
         if (slot >= 0) configured.v[slot] = true;
     }
+    // The register hand-over inside the kernel only ends if the launch really holds kDotsLaunchRegs per thread:
+    // ask what the kernel was built with instead of trusting it.
+    static PerDevice<int> launch_regs;
+    int regs = slot >= 0 ? launch_regs.v[slot] : 0;
+    if (regs == 0) {
+        cudaFuncAttributes attr;
+        cudaError_t e = cudaFuncGetAttributes(&attr, dots_pipe_kernel<NA>);
+        if (e != cudaSuccess) return e;
+        regs = attr.numRegs;
+        if (slot >= 0) launch_regs.v[slot] = regs;
+    }
+    if (regs != kDotsLaunchRegs) return cudaErrorLaunchOutOfResources;
     dots_pipe_kernel<NA><<<grid, kDotsPipeThreads, DotsGeom::kSmemBytes, st>>>(pa);
     return cudaGetLastError();
 }
