@@ -290,7 +290,7 @@ def time_cpu_baseline(cfg, enums, limit_s=12.0, single_thread=True):
            "sample": f"first {d_s} of {cfg['d']} coordinates per step (gradient-stream recipe, same M, K, codec, block), {n} steps, {per * 1e3:.1f} ms each"}
     if single_thread and cores > 1:
         # the same oracle on one thread, on a shorter sample (a quarter of the coordinates, one step)
-        d_1 = max(d_s // 4, 1 << 14)
+        d_1 = min(d_s, max(d_s // 4, 1 << 14))
         orc1 = oracle.State(d_1, M, K, codec, norm, block=cfg["block"], fuse_mode=fuse, qsgd_levels=cfg.get("levels", 7))
         for j in range(K):
             orc1.push_reference(np.ascontiguousarray(orc.history(K - 1 - j)[:d_1]))
@@ -472,6 +472,8 @@ def run_ours(args, name, cfg, emit=True):
         step(w)
     barrier()
     st0 = ctx.stats()
+    if driver is not None:
+        driver.clock.start()        # the split rounds are timed stage by stage by the driver (events between its calls)
     ms_local, clocks = timed_rounds(torch, step, args.steps, barrier, local, flush_buf)
     ms_step = max_over_ranks(ms_local, world, dev)
     st1 = ctx.stats()
@@ -479,13 +481,25 @@ def run_ours(args, name, cfg, emit=True):
 
     peak, peak_src = measured_hbm_peak()
     _, combine_ms = stage_split(st0, st1, {}, d_local, peak, None)
-    ref_in_encode = cfg["norm"] not in ("none", "mean") and cfg["fuse"] != "last" and combine_ms == 0.0
+    # (the rank-local stages of the split rounds run the combine as a pass of its own)
+    ref_in_encode = driver is None and cfg["norm"] not in ("none", "mean") and cfg["fuse"] != "last" and combine_ms == 0.0
     per_coord = algorithmic_bytes_per_coord(M if split != "workers" else M // world, K, bits, cfg["block"], cfg["fuse"],
                                             ref_in_encode=ref_in_encode, norm=cfg["norm"])
     if split == "workers":     # every rank still decodes all M workers' codes
         full = algorithmic_bytes_per_coord(M, K, bits, cfg["block"], cfg["fuse"], ref_in_encode=ref_in_encode, norm=cfg["norm"])
         per_coord["decode"] = full["decode"]
     kernels, _ = stage_split(st0, st1, per_coord, d_local, peak, clocks.get("sm_mhz"))
+    if driver is not None:
+        # rank-local stages: statistics = dots, solve_combine = the solve and the (separate) reference combine
+        stage_ms = driver.clock.times()
+        driver.clock.marks = None
+        kernels = {}
+        for sname, key in (("statistics", "dots"), ("solve_combine", "combine"), ("encode", "encode"), ("decode", "decode")):
+            if key in per_coord and stage_ms.get(sname):
+                ms = stage_ms[sname]
+                gbs = per_coord[key] * d_local / (ms * 1e-3) / 1e9
+                kernels[key] = {"ms": ms, "bytes_per_coord": per_coord[key], "GBps": gbs, "frac_of_measured": gbs / peak}
+        kernels["exchanges"] = {k: v for k, v in stage_ms.items() if k.startswith("exchange")}
     if ref_in_encode and "encode" in kernels:
         kernels["encode"]["includes"] = "reference combine (ring rows -> reference) folded into the encode pass"
     dominant = max((k for k in kernels if "bytes_per_coord" in kernels[k]), key=lambda k: kernels[k]["ms"])
@@ -506,7 +520,7 @@ def run_ours(args, name, cfg, emit=True):
         roofline["alu_pipe"] = {"bound": "alu", "achieved": alu_rate / 1e9, "peak": alu_peak / 1e9, "unit": "G warp-instr/s",
                                 "frac": alu_rate / alu_peak,
                                 "peak_source": "0.5 warp-instr/cycle x 4 partitions x 148 SMs x sampled SM clock"}
-    step_bytes = sum(per_coord.values()) * d_local
+    step_bytes = sum(v for k, v in per_coord.items()) * d_local
     step_gbs = step_bytes / (ms_step * 1e-3) / 1e9
 
     # ---- the same rounds for long enough that the power-limited clock is reached (a short burst runs at the top clock)

@@ -479,17 +479,20 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_kernel(const E
 // The same pass when one scale spans 2, 4, 8 or 16 tiles (blocks of 256 .. 2048
 // coordinates, all inside one chunk): the gradient rows are still read once.  Per fill a
 // warp normalises its tile for the (up to) eight workers, keeps the values in registers and
-// posts the eight tile statistics in shared memory; after a barrier among the compute warps,
-// lane k of every warp combines the statistics of its block for worker k (maximum, or the
-// adjacent-pairwise sum that continues the tree inside the tiles; slots beyond the block count
+// posts the eight tile statistics in shared memory; after a barrier among the warps of the block
+// (each group of 2 .. 16 warps has a hardware barrier of its own, so groups do not wait for one
+// another), lane k of every warp combines the statistics of its block for worker k (maximum, or
+// the adjacent-pairwise sum that continues the tree inside the tiles; slots beyond the block count
 // as zero, the identity of both) and the warp quantises from registers.  Statistics and the
-// give-up flag are double-buffered, so one barrier per fill is enough: a warp can only run one
-// fill ahead of the slowest one.  A warp whose bounded wait runs out raises the flag and still
-// arrives at the fill's barrier; after it all sixteen warps see the flag and leave together,
-// so nobody is left waiting at a barrier.
+// group's give-up flag are double-buffered, so one barrier per fill is enough: a warp can only run
+// one fill ahead of the slowest one of its group.  A warp whose bounded wait runs out raises its
+// group's flag and still arrives at the fill's barrier; after it all warps of the group see the flag
+// and leave together, so nobody is left waiting at a barrier (the other groups then run out of
+// stages, since a stage is only refilled once all sixteen warps have released it, and leave the same way).
 // ---------------------------------------------------------------------------
-__device__ __forceinline__ void compute_warps_barrier() {
-    asm volatile("bar.sync 1, %0;" ::"n"(kEncPipeWarps * 32) : "memory");
+// barrier among the warps of one scale block: hardware barrier 1 + group, `threads` = 32 x warps per block
+__device__ __forceinline__ void block_warps_barrier(const int group, const int threads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(1 + group), "r"(threads) : "memory");
 }
 
 template <int CODEC, int NORM, int SCALE, bool FUSEREF>
@@ -498,10 +501,10 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_blocks_kernel(
     extern __shared__ unsigned char dyn_smem[];
     __shared__ float s_alpha[kMaxK];
     __shared__ float s_stat[2][G::kRows][kEncPipeWarps + 1];
-    __shared__ uint32_t s_gave_up[2];
+    __shared__ uint32_t s_gave_up[kEncPipeWarps / 2][2];   // per group of warps that share a block, per buffer
     const EncodeArgs& a = pa.e;
     if (FUSEREF && threadIdx.x < kMaxK) s_alpha[threadIdx.x] = ((int)threadIdx.x < a.hist_k) ? a.alpha[threadIdx.x] : 0.0f;
-    if (threadIdx.x < 2) s_gave_up[threadIdx.x] = 0u;
+    if (threadIdx.x < kEncPipeWarps) s_gave_up[threadIdx.x / 2][threadIdx.x % 2] = 0u;
     const PipeSmem pipe = pipe_setup<G>(dyn_smem, kEncPipeWarps);   // ends with __syncthreads
     const uint64_t nchunks = a.tile_begin / kEncPipeWarps;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -518,6 +521,7 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_blocks_kernel(
     const uint32_t M = a.M;
     const int tpb = (int)(a.block / kTile);                // tiles per block: 2, 4, 8 or 16
     const int block_warp0 = warp & ~(tpb - 1);             // first warp (tile) of this warp's block within the chunk
+    const int group = warp / tpb;                          // the warps of one block meet on their own barrier
     constexpr int kWords = 4 * CODEC;
     uint32_t it = 0, buf = 0;
     bool alive = true;
@@ -532,7 +536,7 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_blocks_kernel(
             const uint32_t s = it % G::kStages, use = it / G::kStages;
             if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {
                 atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
-                s_gave_up[buf] = 1u;
+                s_gave_up[group][buf] = 1u;
                 alive = false;
                 break;
             }
@@ -565,7 +569,7 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_blocks_kernel(
                 const uint32_t s = it % G::kStages, use = it / G::kStages;
                 if (!__all_sync(kFullMask, mbar_wait(pipe.full(s), use & 1u))) {
                     atomicMax(a.pipe_error, (uint32_t)kPipeFullTimeout);
-                    s_gave_up[buf] = 1u;
+                    s_gave_up[group][buf] = 1u;
                     alive = false;
                 }
                 if (alive) {
@@ -585,26 +589,36 @@ __global__ void __launch_bounds__(kEncPipeThreads, 1) encode_pipe_blocks_kernel(
                     if (lane < G::kRows) s_stat[buf][lane][warp] = my_stat;
                 }
             }
-            compute_warps_barrier();
-            if (s_gave_up[buf] != 0u) return;              // the same answer in all sixteen warps
-            // lane k: the block's statistic for worker k of the fill
-            float bs[kEncPipeWarps];
+            // the first random numbers do not depend on the scale: drawn before the barrier, they fill the wait
+            uint4 x[kPhiloxBatch];
+            philox4x32_10_rk_batch<kPhiloxBatch>(q_lo, q_hi, a.m_base + m0, a.step, a.rk, x);
+            block_warps_barrier(group, tpb * 32);
+            if (s_gave_up[group][buf] != 0u) return;       // the same answer in all warps of the block
+            // lane k: the block's statistic for worker k of the fill (two tiles per block, the common case, apart)
+            const float* mine_stat = &s_stat[buf][lane & (G::kRows - 1)][block_warp0];
+            auto join = [](const float p, const float q) {
+                return (SCALE == 0) ? __uint_as_float(max(__float_as_uint(p), __float_as_uint(q))) : __fadd_rn(p, q);
+            };
+            float block_stat;
+            if (tpb == 2) {
+                block_stat = join(mine_stat[0], mine_stat[1]);
+            } else {
+                float bs[kEncPipeWarps];
 #pragma unroll
-            for (int t = 0; t < kEncPipeWarps; ++t) bs[t] = (t < tpb) ? s_stat[buf][lane & (G::kRows - 1)][block_warp0 + t] : 0.0f;
+                for (int t = 0; t < kEncPipeWarps; ++t) bs[t] = (t < tpb) ? mine_stat[t] : 0.0f;
 #pragma unroll
-            for (int len = kEncPipeWarps; len > 1; len >>= 1)
+                for (int len = kEncPipeWarps; len > 1; len >>= 1)
 #pragma unroll
-                for (int t = 0; t < len / 2; ++t)
-                    bs[t] = (SCALE == 0) ? __uint_as_float(max(__float_as_uint(bs[2 * t]), __float_as_uint(bs[2 * t + 1])))
-                                         : __fadd_rn(bs[2 * t], bs[2 * t + 1]);
-            const float my_R = (SCALE == 0) ? bs[0] : __fsqrt_rn(bs[0]);
+                    for (int t = 0; t < len / 2; ++t) bs[t] = join(bs[2 * t], bs[2 * t + 1]);
+                block_stat = bs[0];
+            }
+            const float my_R = (SCALE == 0) ? block_stat : __fsqrt_rn(block_stat);
             const uint32_t mine = m0 + (uint32_t)lane;
             uint32_t* my_codes = a.codes + ((uint64_t)mine * a.wpw + T * (uint64_t)kWords);
 #pragma unroll
             for (int k0 = 0; k0 < G::kRows; k0 += kPhiloxBatch) {
                 if (m0 + k0 < M) {
-                    uint4 x[kPhiloxBatch];
-                    philox4x32_10_rk_batch<kPhiloxBatch>(q_lo, q_hi, a.m_base + m0 + k0, a.step, a.rk, x);
+                    if (k0 > 0) philox4x32_10_rk_batch<kPhiloxBatch>(q_lo, q_hi, a.m_base + m0 + k0, a.step, a.rk, x);
 #pragma unroll
                     for (int kk = 0; kk < kPhiloxBatch; ++kk) {
                         const int k = k0 + kk;
@@ -870,16 +884,35 @@ __device__ __forceinline__ void decode_worker(const uint32_t (&w)[4 * CODEC], co
                 : "r"(w[c]), "r"(pw), "r"(okm), "r"(Re));
         }
     } else {
-        const float step = __fdiv_rn(R, (float)levels);
+        // R is what slot_scale left in the slot: the quantiser's step R / s, or NaN for an unusable scale
+        const float step = R;
+        const uint32_t signmask = (step == step) ? 0x80000000u : 0u;
+        const float stepq = (step == step) ? step : 0.0f;
+        // the lane's bit of the three level planes, landed at bit 0, 1 and 2 by a shift and two rotations and
+        // merged by bit-select operations: six instructions per coordinate
+        const uint32_t rot1 = (uint32_t)(lane - 1) & 31u, rot2 = (uint32_t)(lane - 2) & 31u;
 #pragma unroll
         for (int c = 0; c < 4; ++c) {
-            const uint32_t L = ((w[c * 4] >> lane) & 1u) | (((w[c * 4 + 1] >> lane) & 1u) << 1) |
-                               (((w[c * 4 + 2] >> lane) & 1u) << 2);
-            const float mag = __fmul_rn((float)L, step);
-            const float vh = ok ? __uint_as_float(__float_as_uint(mag) ^ ((w[c * 4 + 3] * pw) & 0x80000000u)) : 0.0f;
+            const uint32_t x0 = w[c * 4] >> lane;
+            const uint32_t x1 = __funnelshift_r(w[c * 4 + 1], w[c * 4 + 1], rot1);
+            const uint32_t x2 = __funnelshift_r(w[c * 4 + 2], w[c * 4 + 2], rot2);
+            const uint32_t y = (x0 & 1u) | (x1 & ~1u);
+            const uint32_t L = ((y & 3u) | (x2 & ~3u)) & 7u;
+            const float mag = __fmul_rn((float)L, stepq);
+            const float vh = __uint_as_float(__float_as_uint(mag) ^ ((w[c * 4 + 3] * pw) & signmask));
             acc[c] = __fadd_rn(acc[c], vh);
         }
     }
+}
+
+// What goes into the decode slot for a worker's scale.  Ternary and sign codes use the scale as it is.  The
+// s-level quantiser needs the step R / s (one IEEE division): taken here once per worker and tile by the lane that
+// fetched the scale, instead of by every lane for every worker; an unusable scale (zero, NaN, infinite) becomes NaN.
+template <int CODEC>
+__device__ __forceinline__ float slot_scale(const float R, const int levels) {
+    if (CODEC != TNG_CODEC_QSGD4) return R;
+    const bool ok = (__float_as_uint(R) - 1u) < 0x7f7fffffu;
+    return ok ? __fdiv_rn(R, (float)levels) : __int_as_float(0x7fc00000);
 }
 
 // average over the M workers (Algorithm 1), put the reference back (Eq. 2 / Eq. 3), store
@@ -1043,7 +1076,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
     if (T < nfull) fetch(T, cw, sc, r, r2);
     for (; T < nfull; T += nwarps) {
         slot->cw[lane] = cw;
-        slot->sc[lane] = sc;
+        slot->sc[lane] = slot_scale<CODEC>(sc, a.levels);
         const float4 rcur = r, r2cur = r2;
         __syncwarp();
         const uint32_t Tn = T + nwarps;
@@ -1056,7 +1089,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
             decode_fetch<CODEC>(a, T, tiled ? T : ((uint64_t)T * kTile) / a.block, m0, lane, cw2, sc2);
             __syncwarp();
             slot->cw[lane] = cw2;
-            slot->sc[lane] = sc2;
+            slot->sc[lane] = slot_scale<CODEC>(sc2, a.levels);
             __syncwarp();
             decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
         }
@@ -1080,7 +1113,7 @@ __global__ void __launch_bounds__(kCodecThreads, 4) decode_kernel(const DecodeAr
             decode_fetch<CODEC>(a, Tr, blk, m0, lane, cw2, sc2);
             __syncwarp();
             slot->cw[lane] = cw2;
-            slot->sc[lane] = sc2;
+            slot->sc[lane] = slot_scale<CODEC>(sc2, a.levels);
             __syncwarp();
             decode_round<CODEC>(slot, (a.M - m0 < kRound) ? a.M - m0 : kRound, a.levels, pw, lane, acc);
         }

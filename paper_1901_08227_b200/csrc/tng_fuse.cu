@@ -368,7 +368,7 @@ cudaError_t dots_cross_n(int n, const DotsArgs& a, int grid, cudaStream_t st) {
 //
 // Lane i owns row i of the augmented system [A | b] in shared memory.  Elimination is
 // right-looking: at step j every lane below the pivot scales its entry of column j by the
-// pivot's root, then subtracts the rank-one term from the rest of its row and from its b.
+// reciprocal of the pivot's root, then subtracts the rank-one term from the rest of its row and from its b.
 // When the sweep ends column n holds the forward-substituted right-hand side, so only the
 // backward sweep (column by column, again one lane per row) remains.  A pivot that is not a
 // finite positive number above 1e-12 of the diagonal entry it started from is rounding
@@ -386,10 +386,12 @@ __device__ bool warp_spd_solve(double* S, double* x, const int n, const int lane
         const double piv = S[j * kSolveLd + j];
         const double ref = __shfl_sync(kFullMask, start_diag, j);
         if (!(piv > 1e-12 * ref) || !(piv > 0.0) || !isfinite(piv)) { good = false; break; }   // the same in all lanes
-        const double root = sqrt(piv);
+        // one reciprocal square root per pivot; everything else multiplies by it (the diagonal keeps 1/root,
+        // which is what the backward sweep needs)
+        const double rinv = rsqrt(piv);
         __syncwarp();
-        if (lane >= j && lane < n) S[lane * kSolveLd + j] = (lane == j) ? root : S[lane * kSolveLd + j] / root;
-        if (lane == j) S[j * kSolveLd + n] /= root;
+        if (lane >= j && lane < n) S[lane * kSolveLd + j] = (lane == j) ? rinv : S[lane * kSolveLd + j] * rinv;
+        if (lane == j) S[j * kSolveLd + n] *= rinv;
         __syncwarp();
         if (lane > j && lane < n) {
             const double mine = S[lane * kSolveLd + j];
@@ -401,7 +403,7 @@ __device__ bool warp_spd_solve(double* S, double* x, const int n, const int lane
     if (!good) return false;
     // backward sweep on L^T: the newest unknown is final, every lane above it removes its share
     for (int i = n - 1; i >= 0; --i) {
-        if (lane == i) S[i * kSolveLd + n] /= S[i * kSolveLd + i];
+        if (lane == i) S[i * kSolveLd + n] *= S[i * kSolveLd + i];   // the diagonal holds 1/root
         __syncwarp();
         if (lane < i) S[lane * kSolveLd + n] -= S[i * kSolveLd + lane] * S[i * kSolveLd + n];
         __syncwarp();

@@ -31,14 +31,47 @@ def worker_range(rank: int, world: int, M: int):
     return rank * count, count
 
 
+class _StageClock:
+    """Optional CUDA-event marks between the stages of a round (on the current stream, which is the one
+    the library calls are given): mean milliseconds per stage over the rounds since start_timing()."""
+
+    def __init__(self, names):
+        self.names, self.marks = names, None
+
+    def start(self):
+        self.marks = []
+
+    def mark(self):
+        if self.marks is not None:
+            ev = torch.cuda.Event(enable_timing=True)
+            ev.record()
+            self.marks.append(ev)
+
+    def times(self):
+        n = len(self.names) + 1
+        if not self.marks or len(self.marks) < n:
+            return {}
+        torch.cuda.synchronize()
+        rounds = len(self.marks) // n
+        out = {name: 0.0 for name in self.names}
+        for r in range(rounds):
+            evs = self.marks[r * n:(r + 1) * n]
+            for i, name in enumerate(self.names):
+                out[name] += evs[i].elapsed_time(evs[i + 1]) / rounds
+        return out
+
+
 class DistributedRound:
     """Drives one context per rank.  `group` may be None (a single process: no exchange)."""
+
+    STAGES = ("statistics", "exchange_statistics", "solve_combine", "encode", "exchange_wire", "decode")
 
     def __init__(self, ctx: tng.Context, group=None):
         self.ctx, self.group = ctx, group
         self.world = dist.get_world_size(group) if group is not None else 1
         self.rank = dist.get_rank(group) if group is not None else 0
         self.first, self.count = worker_range(self.rank, self.world, ctx.M)
+        self.clock = _StageClock(self.STAGES)
         self.resync()
 
     def resync(self):
@@ -50,14 +83,20 @@ class DistributedRound:
         """local_grads: (count, d) rows of this rank's workers.  Returns `out` (the aggregate)."""
         if local_grads.shape[0] != self.count:
             raise ValueError(f"rank {self.rank} owns {self.count} workers, got {local_grads.shape[0]} rows")
-        ctx = self.ctx
+        ctx, clock = self.ctx, self.clock
         scalar_ref = ctx.norm == tng.NORM_MEAN          # every worker's own scalar: no fusion, no statistics
+        clock.mark()
         if not scalar_ref:
             ctx.fuse_local(local_grads)
-            if self.world > 1:
-                dist.all_reduce(ctx.local_stats(), op=dist.ReduceOp.SUM, group=self.group)
+        clock.mark()
+        if not scalar_ref and self.world > 1:
+            dist.all_reduce(ctx.local_stats(), op=dist.ReduceOp.SUM, group=self.group)
+        clock.mark()
+        if not scalar_ref:
             ctx.fuse_finish()
+        clock.mark()
         ctx.encode_local(local_grads, self.first, self.round)
+        clock.mark()
         if self.world > 1:
             codes, scales = ctx.wire_views()
             lo, hi = self.first, self.first + self.count
@@ -66,7 +105,9 @@ class DistributedRound:
             if scalar_ref:                               # the scalars travel with the codes
                 means = ctx.wire_means_view()
                 dist.all_gather_into_tensor(means, means[lo:hi].clone(), group=self.group)
+        clock.mark()
         ctx.decode_commit(out)
+        clock.mark()
         self.round += 1
         return out
 
@@ -96,9 +137,12 @@ class CoordShardedRound:
 
     Every rank ends up with its slice of what one context over the whole vector computes."""
 
+    STAGES = ("statistics", "exchange_statistics", "solve_combine", "encode", "decode")
+
     def __init__(self, ctx: tng.Context, group=None):
         self.ctx, self.group = ctx, group
         self.world = dist.get_world_size(group) if group is not None else 1
+        self.clock = _StageClock(self.STAGES)
         self.resync()
 
     def resync(self):
@@ -110,11 +154,18 @@ class CoordShardedRound:
         ctx = self.ctx
         if grads_slice.shape[0] != ctx.M:
             raise ValueError(f"expected the rows of all {ctx.M} workers, got {grads_slice.shape[0]}")
+        clock = self.clock
+        clock.mark()
         ctx.fuse_local(grads_slice)
+        clock.mark()
         if self.world > 1:
             dist.all_reduce(ctx.local_stats_all(), op=dist.ReduceOp.SUM, group=self.group)
+        clock.mark()
         ctx.fuse_finish()
+        clock.mark()
         ctx.encode_local(grads_slice, 0, self.round)
+        clock.mark()
         ctx.decode_commit(out)
+        clock.mark()
         self.round += 1
         return out
