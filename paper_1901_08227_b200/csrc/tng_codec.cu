@@ -719,6 +719,32 @@ __global__ void __launch_bounds__(256) block_scale_level_kernel(const float* __r
     }
 }
 
+// The same reduction for blocks of at most 32 tiles (there can be millions of them): one warp per (block,
+// worker), a lane per tile, xor-shuffles pair neighbouring lanes.  Zero-padding to 32 entries instead of to the
+// next power of two only appends additions of zero (or maxima with zero), so the value is the same.
+template <int SCALE>
+__global__ void __launch_bounds__(256) block_scale_warp_kernel(const float* __restrict__ in, uint64_t n_in, uint32_t seg,
+                                                               float* __restrict__ out, uint64_t n_out, uint64_t nblk,
+                                                               uint32_t M, unsigned long long* nonfinite) {
+    const int lane = threadIdx.x & 31;
+    const uint64_t nwarps = (uint64_t)gridDim.x * 8u;
+    for (uint64_t job = (uint64_t)blockIdx.x * 8u + (threadIdx.x >> 5); job < nblk * M; job += nwarps) {
+        const uint64_t m = job / nblk, blk = job % nblk;
+        const uint64_t t = blk * seg + (uint32_t)lane;
+        float x = ((uint32_t)lane < seg && t < n_in) ? in[m * n_in + t] : 0.0f;
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float y = __shfl_xor_sync(kFullMask, x, off);
+            x = (SCALE == 0) ? __uint_as_float(max(__float_as_uint(x), __float_as_uint(y))) : __fadd_rn(x, y);
+        }
+        if (lane == 0) {
+            const float r = (SCALE == 1) ? __fsqrt_rn(x) : x;
+            if (!(fabsf(r) < __int_as_float(0x7f800000))) atomicAdd(nonfinite, 1ull);
+            out[m * n_out + blk] = r;
+        }
+    }
+}
+
 // ---------------------------------------------------------------------------
 // Short problems (a per-vector scale at small d, odd block sizes of short vectors): the three
 // launches statistic -> tree -> quantise are latency, not bandwidth.  Here one CTA owns one
@@ -1437,6 +1463,19 @@ cudaError_t launch_encode(const CodecGeom& g, uint32_t m_base, const float* grad
     uint64_t seg = (g.block + kTile - 1) / kTile;
     float* ping = tree_tmp;
     float* pong = tree_tmp + tree_tmp_floats(g) / 2;
+    if (seg <= 32) {   // small blocks: a warp per block instead of a CTA per block
+        const uint64_t jobs = nblk_rest * (uint64_t)g.M;
+        const uint64_t want = (jobs + 7) / 8, cap = (uint64_t)sm_count * 16u;
+        const unsigned grid = (unsigned)(want < cap ? want : cap);
+        if (g.scale_kind == 0)
+            block_scale_warp_kernel<0><<<grid, 256, 0, st>>>(in, n_in, (uint32_t)seg, a.scales, g.nblk, nblk_rest, g.M, &fb->nonfinite);
+        else
+            block_scale_warp_kernel<1><<<grid, 256, 0, st>>>(in, n_in, (uint32_t)seg, a.scales, g.nblk, nblk_rest, g.M, &fb->nonfinite);
+        ++*launches;
+        e = cudaGetLastError();
+        if (e != cudaSuccess) return e;
+        return encode_dispatch(a, g.codec, g.norm, g.scale_kind, kPhaseQuant, sm_count, st, launches);
+    }
     for (;;) {
         const uint64_t chunks = (seg + 1023) / 1024;
         const int final = chunks == 1;
