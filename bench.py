@@ -481,8 +481,8 @@ def run_ours(args, name, cfg, emit=True):
 
     peak, peak_src = measured_hbm_peak()
     _, combine_ms = stage_split(st0, st1, {}, d_local, peak, None)
-    # (the rank-local stages of the split rounds run the combine as a pass of its own)
-    ref_in_encode = driver is None and cfg["norm"] not in ("none", "mean") and cfg["fuse"] != "last" and combine_ms == 0.0
+    # (in the rank-local rounds the first tng_encode_local after a fusion forms the reference, as tng_step's encode does)
+    ref_in_encode = cfg["norm"] not in ("none", "mean") and cfg["fuse"] != "last" and (driver is not None or combine_ms == 0.0)
     per_coord = algorithmic_bytes_per_coord(M if split != "workers" else M // world, K, bits, cfg["block"], cfg["fuse"],
                                             ref_in_encode=ref_in_encode, norm=cfg["norm"])
     if split == "workers":     # every rank still decodes all M workers' codes
@@ -490,15 +490,16 @@ def run_ours(args, name, cfg, emit=True):
         per_coord["decode"] = full["decode"]
     kernels, _ = stage_split(st0, st1, per_coord, d_local, peak, clocks.get("sm_mhz"))
     if driver is not None:
-        # rank-local stages: statistics = dots, solve_combine = the solve and the (separate) reference combine
+        # rank-local stages: statistics = dots, solve_combine = tng_fuse_finish (the solve; the combine is left to the encode)
         stage_ms = driver.clock.times()
         driver.clock.marks = None
         kernels = {}
-        for sname, key in (("statistics", "dots"), ("solve_combine", "combine"), ("encode", "encode"), ("decode", "decode")):
+        for sname, key in (("statistics", "dots"), ("encode", "encode"), ("decode", "decode")):
             if key in per_coord and stage_ms.get(sname):
                 ms = stage_ms[sname]
                 gbs = per_coord[key] * d_local / (ms * 1e-3) / 1e9
                 kernels[key] = {"ms": ms, "bytes_per_coord": per_coord[key], "GBps": gbs, "frac_of_measured": gbs / peak}
+        kernels["solve"] = {"ms": stage_ms.get("solve_combine", 0.0)}
         kernels["exchanges"] = {k: v for k, v in stage_ms.items() if k.startswith("exchange")}
     if ref_in_encode and "encode" in kernels:
         kernels["encode"]["includes"] = "reference combine (ring rows -> reference) folded into the encode pass"

@@ -208,7 +208,9 @@ tng_status tng_decode_aggregate(tng_ctx* ctx, const float* ref_dev, float* out_d
  *   tng_fuse_local      statistics of the local rows: Gram of the ring (the same on every rank)
  *                       and the local SUMS sum_m <h_i, g^m>, sum_m ||g^m||^2
  *   [all-reduce (sum) of the tng_local_stats block: 17 doubles on the device]
- *   tng_fuse_finish     divide by M, solve, combine -> the reference (Sec. 3.1 / Prop. 2)
+ *   tng_fuse_finish     divide by M, solve -> the coefficients of the reference (Sec. 3.1 / Prop. 2); the
+ *                       combine itself is done by the pass of the next tng_encode_local, which reads the
+ *                       ring anyway (or, should another call need the reference first, by that call)
  *   tng_encode_local    code the local rows as workers m_first.. into THEIR slots of the wire
  *   [all-gather of the wire: every rank's slots of codes and scales (tng_wire)]
  *   tng_decode_commit   decode all M workers, average, put the reference back, push into the

@@ -52,6 +52,10 @@ struct tng_ctx {
     bool last_had_stats = false;
     bool last_solved = false;         // the last fusion ran the solve kernel (alpha lives on the device)
     bool ref2_valid = false;          // combined form: the second-reference buffer has been written
+    // rank-local rounds: tng_fuse_finish leaves the combine r = sum alpha_j h_j to the next tng_encode_local (which
+    // reads the ring rows anyway); any other reader of the reference has it formed first (materialise_ref)
+    bool ref_pending = false;
+    RefFusion pending{};
     // bookkeeping
     int device = 0, sm_count = 148;
     cudaStream_t last_stream = nullptr;
@@ -281,9 +285,21 @@ tng_status do_decode(tng_ctx* c, const float* ref, float* out_a, float* out_b, c
     return TNG_OK;
 }
 
+// Form the reference a rank-local fusion left to the encode pass, if it is still owed.
+tng_status materialise_ref(tng_ctx* c, cudaStream_t st) {
+    if (!c->ref_pending) return TNG_OK;
+    int launches = 0;
+    TNG_CUDA(c, launch_combine(c->pending.rows, c->pending.k, c->d, c->fb(), c->ref_buf(), c->ref2_buf(), c->sm_count, st, &launches));
+    c->launches += (uint64_t)launches;
+    c->ref_pending = false;
+    return TNG_OK;
+}
+
 // The decoded aggregate goes straight into the next ring slot (and to the caller's buffer); the
 // round is then complete: ring rotated, round counter advanced.
 tng_status decode_commit(tng_ctx* c, float* out, cudaStream_t st) {
+    tng_status sm = materialise_ref(c, st);
+    if (sm != TNG_OK) return sm;
     const int slot = (c->k == 0) ? c->head : (c->head + 1) % (int)c->K;
     tng_status s = do_decode(c, c->ref_cur, c->ring(slot), out, st);
     if (s != TNG_OK) return s;
@@ -294,6 +310,10 @@ tng_status decode_commit(tng_ctx* c, float* out, cudaStream_t st) {
 }
 
 tng_status step_impl(tng_ctx* c, const float* grads, uint64_t ld, float* out, cudaStream_t st) {
+    {
+        tng_status sm = materialise_ref(c, st);   // (a held reference may still be owed by a rank-local fusion)
+        if (sm != TNG_OK) return sm;
+    }
     StageTimer tm(c, st);
     RefFusion fusion;
     fusion.k = 0;
@@ -434,6 +454,8 @@ tng_status tng_push_reference(tng_ctx* c, const float* vec_dev, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     tng_status s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
+    s = materialise_ref(c, st);   // the slot written below may be a row an owed combine still reads
+    if (s != TNG_OK) return s;
     const int slot = (c->k == 0) ? c->head : (c->head + 1) % (int)c->K;
     TNG_CUDA(c, cudaMemcpyAsync(c->ring(slot), vec_dev, c->d * sizeof(float), cudaMemcpyDeviceToDevice, st));
     c->head = slot;
@@ -541,6 +563,8 @@ tng_status tng_save_state(tng_ctx* c, void* host_buf, size_t bytes, size_t* writ
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     tng_status s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
+    s = materialise_ref(c, st);
+    if (s != TNG_OK) return s;
     StateHeader h;
     fill_header(c, &h);
     h.has_ref = (c->ref_every > 1 && c->ref_cur) ? 1u : 0u;
@@ -584,6 +608,7 @@ tng_status tng_load_state(tng_ctx* c, const void* host_buf, size_t bytes, void* 
     if (h.has_ref == 2) TNG_CUDA(c, cudaMemcpyAsync(c->ref2_buf(), p + vec, vec, cudaMemcpyHostToDevice, st));
     TNG_CUDA(c, cudaStreamSynchronize(st));
     c->ref2_valid = h.has_ref == 2;
+    c->ref_pending = false;
     c->k = h.k;
     c->head = h.k ? (int)h.k - 1 : 0;
     c->rounds = h.rounds;
@@ -655,7 +680,10 @@ tng_status tng_fuse_finish(tng_ctx* c, void* stream) {
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     tng_status s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
-    return do_fuse(c, nullptr, 0, st, nullptr, nullptr, true);
+    c->ref_pending = false;
+    s = do_fuse(c, nullptr, 0, st, nullptr, &c->pending, true);
+    if (s == TNG_OK && c->pending.k > 0) c->ref_pending = true;
+    return s;
 }
 
 tng_status tng_encode_local(tng_ctx* c, const float* grads_dev, uint64_t ld, uint32_t m_first, uint32_t m_count, uint32_t step,
@@ -671,7 +699,9 @@ tng_status tng_encode_local(tng_ctx* c, const float* grads_dev, uint64_t ld, uin
     CodecGeom g = c->geom;
     g.M = m_count;
     int launches = 0;
-    TNG_CUDA(c, launch_encode(g, m_first, grads_dev, ld, c->ref_cur, c->ref2_buf(), nullptr, step, c->codes() + (size_t)m_first * g.wpw,
+    const RefFusion* owed = c->ref_pending ? &c->pending : nullptr;   // the first encode after a fusion forms the reference
+    c->ref_pending = false;
+    TNG_CUDA(c, launch_encode(g, m_first, grads_dev, ld, c->ref_cur, c->ref2_buf(), owed, step, c->codes() + (size_t)m_first * g.wpw,
                               c->scales() + (size_t)m_first * g.nblk, c->means() + m_first, c->tile_stat(), c->tree(), c->fb(),
                               c->sm_count, st, &launches));
     c->launches += (uint64_t)launches;
@@ -695,6 +725,7 @@ tng_status tng_fuse(tng_ctx* c, const float* grads_dev, uint64_t ld, void* strea
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     s = ensure_ready(c, st);
     if (s != TNG_OK) return s;
+    c->ref_pending = false;   // a new fusion replaces whatever reference was still owed
     return do_fuse(c, grads_dev, ld, st, nullptr, nullptr);
 }
 
@@ -705,6 +736,8 @@ tng_status tng_encode(tng_ctx* c, const float* grads_dev, uint64_t ld, const flo
     if (ref_dev && !aligned16(ref_dev)) return TNG_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    s = materialise_ref(c, st);
     if (s != TNG_OK) return s;
     const float* ref = ref_dev ? ref_dev : c->ref_cur;
     if (!ref && !c->no_ref()) return TNG_ERR_STATE;   // no fusion has produced a reference yet
@@ -717,6 +750,8 @@ tng_status tng_decode_aggregate(tng_ctx* c, const float* ref_dev, float* out_dev
     if (ref_dev && !aligned16(ref_dev)) return TNG_ERR_INVALID_ARG;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     tng_status s = ensure_ready(c, st);
+    if (s != TNG_OK) return s;
+    s = materialise_ref(c, st);
     if (s != TNG_OK) return s;
     const float* ref = ref_dev ? ref_dev : c->ref_cur;
     if (!ref && !c->no_ref()) return TNG_ERR_STATE;
@@ -745,6 +780,7 @@ tng_status tng_wire_means(tng_ctx* c, const float** means_dev) {
 tng_status tng_reference(tng_ctx* c, const float** ref_dev) {
     if (!c || !ref_dev) return TNG_ERR_INVALID_ARG;
     if (!c->ws_ready || !c->ref_cur) return TNG_ERR_STATE;
+    if (materialise_ref(c, c->last_stream) != TNG_OK) return TNG_ERR_CUDA;   // on the stream of the last call
     *ref_dev = c->ref_cur;
     return TNG_OK;
 }
