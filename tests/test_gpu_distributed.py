@@ -214,3 +214,40 @@ def test_a_slice_needs_whole_blocks_and_no_whole_vector_quantities():
     assert distributed.coord_range(1, 2, 1000, 128) == (512, 488)
     with pytest.raises(ValueError):
         distributed.coord_range(3, 4, 300, 128)
+
+
+@pytest.mark.parametrize("reader", ["reference", "save_state", "decode", "encode_in_two_calls"])
+def test_a_reference_still_owed_after_fuse_finish_is_formed_by_whoever_needs_it_first(reader):
+    # tng_fuse_finish leaves r = sum alpha_j h_j to the next tng_encode_local.  Whatever else touches the
+    # reference first (reading it, saving the state, decoding, an encode of only some of the workers followed by
+    # another) must see the same reference and produce the same round as the plain order of calls.
+    d, M, K = 2048 * 9 + 128 * 3 + 8, 8, 3
+    opts = dict(block=128, fuse_mode=tng.FUSE_MEAN, seed_lo=12)
+    a = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_DIFF, **opts)      # plain order
+    b = make_ctx(d, M, K, tng.CODEC_TERN2, tng.NORM_DIFF, **opts)      # with the extra reader
+    oa, ob = torch.empty(d, device="cuda"), torch.empty(d, device="cuda")
+    for t, g in enumerate(drifting_grads(14, K + 3, M, d, "cuda")):
+        a.fuse_local(g)
+        a.fuse_finish()
+        a.encode_local(g, 0, t)
+        a.decode_commit(oa)
+        b.fuse_local(g)
+        b.fuse_finish()
+        if reader == "reference" and t > 0:
+            early = b.reference()
+        elif reader == "save_state":
+            b.save_state()
+        elif reader == "decode" and t > 0:
+            b.decode_aggregate(ob)                      # decodes the previous wire against the new reference: only must not fault
+        if reader == "encode_in_two_calls":
+            b.encode_local(g[:3], 0, t)
+            b.encode_local(g[3:], 3, t)
+        else:
+            b.encode_local(g, 0, t)
+        b.decode_commit(ob)
+        assert torch.equal(oa, ob), f"round {t}"
+        assert torch.equal(a.wire()[0], b.wire()[0]) and torch.equal(a.wire()[1], b.wire()[1])
+        assert torch.equal(a.reference(), b.reference())
+        if reader == "reference" and t > 0:
+            assert torch.equal(early, b.reference())
+    assert a.stats().rounds == b.stats().rounds == K + 3
