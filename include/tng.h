@@ -67,7 +67,10 @@ typedef enum {
 
 typedef enum {
     TNG_OPT_BLOCK = 0,       /* coordinates per scale; 0 = one scale per vector (the paper's R);
-                                otherwise a multiple of 128.  Default 128. */
+                                otherwise a multiple of 128.  Default 128.  Cost: 128, 256, 512, 1024 and 2048
+                                are encoded in one read of the gradient rows; any other value (0 included)
+                                needs the scale before the first symbol, i.e. two reads, except for short
+                                problems (tiles x workers <= 16384), which are one launch either way. */
     TNG_OPT_QSGD_LEVELS = 1, /* s in 1..7 (TNG_CODEC_QSGD4 only).  Default 7. */
     TNG_OPT_SCALE_KIND = 2,  /* 0 = max|v| (Sec. 3.2), 1 = L2 norm of the block.  Default 0. */
     TNG_OPT_SEED_LO = 3,     /* low / high 32 bits of the Philox key.  Default 0. */
